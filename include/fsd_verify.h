@@ -1,0 +1,153 @@
+/*
+ * fsd_verify.h -- C ABI of the batched verification step of Fuzzy Speculative
+ * Decoding (FSD) and of strict speculative sampling (SD) on one NVIDIA B200.
+ *
+ * What a call computes, for every batch row b and candidate position i:
+ *   1. P_T[i] = softmax(target_logits[b, i, :]), P_D[i] = softmax(draft_logits[b, i, :])
+ *      (Section 4: "next token distributions at candidate position i").
+ *   2. The divergence D[b, i] = Div(P_T[i], P_D[i]) in nats: Jensen-Shannon
+ *      (Appendix C.2, the paper's default), KL(P_T || P_D) (Appendix C.1) or total
+ *      variation (Appendix C.3).
+ *   3. The acceptance bit: FSD accepts iff D < T (Section 4, Eq. 4; "<=" selectable);
+ *      SD accepts iff u_accept < min(1, P_T(x_i)/P_D(x_i)) (Section 3, Eq. 1-2);
+ *      rFSD accepts iff either holds (Section 4.3, Eq. 6).
+ *   4. accept_len[b] = index of the first rejected position, or gamma (Section 3,
+ *      "first rejection").
+ *   5. next_token[b]: FSD draws it from P_T at the rejected position (Section 4);
+ *      SD and rFSD from max(0, P_T - P_D) renormalised (Section 3, Eq. 3); when every
+ *      candidate was accepted it is drawn from P_T of the extra row gamma.  The draw
+ *      is the inverse CDF in vocabulary order at u_sample[b] (smallest k whose
+ *      cumulative weight exceeds u * total), or the argmax when FSD_SAMPLE_GREEDY
+ *      (Section 6.3).
+ * fsd_verify_tree applies the same per-node test to a draft tree (Section 6.4) and
+ * returns the deepest root-to-node path whose nodes all pass.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a parameter says
+ *     "host".  The library allocates no device memory: scratch space is the caller's
+ *     `workspace`, sized by fsd_workspace_bytes().
+ *   - Logit tensors are row-major and contiguous, both of the dtype named in the
+ *     options.  Rows whose byte length is a multiple of 16 with 16-byte aligned bases
+ *     take the vectorised kernels; any other shape takes a slower scalar kernel.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream).  Outputs are valid once the stream has been synchronised.
+ *   - The return value is a host-side status: FSD_OK (0) or a negative FSD_ERR_*.
+ *     On error nothing has been launched.  Nothing aborts, throws or traps.
+ *   - Conditions found on the device are reported per batch row in row_status.
+ *   - -inf logits are legal (probability zero).  A row holding NaN, +inf or no finite
+ *     value makes its position's divergence NaN, rejects the position and sets
+ *     FSD_ROW_NONFINITE.
+ */
+#ifndef FSD_VERIFY_H
+#define FSD_VERIFY_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* divergence (Appendix C) */
+#define FSD_DIV_JS 0
+#define FSD_DIV_KL 1   /* KL(P_T || P_D) */
+#define FSD_DIV_TV 2
+/* acceptance rule */
+#define FSD_MODE_FSD  0 /* Section 4, Eq. 4 */
+#define FSD_MODE_SD   1 /* Section 3, Eq. 1-3 */
+#define FSD_MODE_RFSD 2 /* Section 4.3, Eq. 6 */
+/* threshold comparison */
+#define FSD_CMP_LT 0    /* accept iff D <  T (as printed in Eq. 4) */
+#define FSD_CMP_LE 1    /* accept iff D <= T */
+/* replacement-token choice */
+#define FSD_SAMPLE_INVCDF 0
+#define FSD_SAMPLE_GREEDY 1 /* Section 6.3 */
+/* logit storage */
+#define FSD_F32  0
+#define FSD_BF16 1
+
+/* host status codes */
+#define FSD_OK               0
+#define FSD_ERR_NULL        -1  /* a required pointer is NULL */
+#define FSD_ERR_SHAPE       -2  /* B < 1, gamma/N < 1, V < 1, max_depth < 1, or a size overflows */
+#define FSD_ERR_ALIGN       -3  /* a pointer is not aligned to its element size (workspace: 256 bytes) */
+#define FSD_ERR_ENUM        -4  /* an option value is out of range, or struct_size is wrong */
+#define FSD_ERR_WORKSPACE   -5  /* workspace_bytes is smaller than fsd_workspace_bytes() reports */
+#define FSD_ERR_UNSUPPORTED -6  /* combination not defined (SD / rFSD on a tree) */
+#define FSD_ERR_CUDA        -7  /* the CUDA runtime refused a launch or a copy */
+
+/* row_status bit flags (device-side conditions) */
+#define FSD_ROW_NONFINITE 1  /* some logit row read for this batch row was not a valid distribution */
+#define FSD_ROW_TIMEOUT   2  /* a bounded device-side wait ran out; outputs of the row are not valid */
+#define FSD_ROW_BADTREE   4  /* parent[] violated -1 <= parent[j] < j */
+
+typedef struct fsd_opts {
+    uint32_t struct_size;  /* sizeof(fsd_opts), for versioning */
+    int32_t  divergence;   /* FSD_DIV_*    */
+    int32_t  mode;         /* FSD_MODE_*   */
+    int32_t  compare;      /* FSD_CMP_*    */
+    int32_t  sample;       /* FSD_SAMPLE_* */
+    int32_t  logit_dtype;  /* FSD_F32 | FSD_BF16 (both tensors) */
+    float    threshold;    /* T of Eq. 4, in nats */
+} fsd_opts;
+
+/* Fills `opts` with the defaults: JS divergence, FSD rule, "<", inverse-CDF sampling,
+ * bf16 logits, T = 0.  Host pointer. */
+void fsd_default_opts(fsd_opts *opts);
+
+/* Bytes of device scratch the verify calls need for B batch rows of `positions`
+ * candidates each (gamma for a chain, N for a tree).  `bytes_out` is a host pointer.
+ * Returns FSD_OK or FSD_ERR_NULL / FSD_ERR_SHAPE / FSD_ERR_ENUM. */
+int fsd_workspace_bytes(int B, int positions, int V, const fsd_opts *opts, size_t *bytes_out);
+
+/* Chain verification (Sections 3 and 4).
+ *   target_logits [B, gamma+1, V]  row i scores candidate i; row gamma supplies the bonus token
+ *   draft_logits  [B, gamma,   V]
+ *   draft_tokens  [B, gamma] int32 candidate ids x_i; may be NULL when mode == FSD_MODE_FSD.
+ *                 An id outside [0, V) is rejected by the ratio test.
+ *   u_accept      [B, gamma] float uniforms in [0,1) for the ratio test; may be NULL in FSD mode
+ *   u_sample      [B]        float uniforms in [0,1) for the one token drawn per row
+ *   opts          host pointer
+ *   accept_len    [B] out    n in [0, gamma]
+ *   next_token    [B] out    token id, or -1 if the row it is drawn from is not a valid distribution
+ *   divergence    [B, gamma] out, float, computed for every position in every mode
+ *   row_status    [B] out    FSD_ROW_* flags
+ *   workspace     device scratch, 256-byte aligned, at least fsd_workspace_bytes() bytes;
+ *                 contents need not be initialised and are not preserved
+ * Calls that share a workspace must be ordered on the stream(s) that use it. */
+int fsd_verify_chain(const void *target_logits, const void *draft_logits,
+                     const int32_t *draft_tokens, const float *u_accept, const float *u_sample,
+                     int B, int gamma, int V, const fsd_opts *opts,
+                     int32_t *accept_len, int32_t *next_token, float *divergence, int32_t *row_status,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* Tree verification (Section 6.4; the paper states no rule, this is the reading used).
+ *   target_logits [B, N+1, V]  row 0 = distribution after the root context, row j+1 = after node j
+ *   draft_logits  [B, N,   V]  row j = distribution node j's token was proposed from
+ *   parent        [B, N] int32  parent[j] in [-1, j); -1 = child of the root
+ *   u_sample      [B]
+ *   max_depth     width of `path`; nodes deeper than max_depth are not eligible
+ *   accept_len    [B] out     depth of the chosen node (0 = nothing accepted)
+ *   path          [B, max_depth] out  node ids from the root's child down to the chosen node, -1 padded
+ *   next_token    [B] out     drawn from the target row after the chosen node (row 0 if none)
+ *   divergence    [B, N] out  Div(P_T[row parent(j)+1], P_D[row j])
+ * Node j passes iff its divergence passes the threshold test; it is on an accepted path iff it
+ * and all its ancestors pass; the chosen node is the deepest such node, ties to the lowest index.
+ * Only FSD_MODE_FSD is defined for trees (others: FSD_ERR_UNSUPPORTED).  A row whose parent
+ * array is invalid gets FSD_ROW_BADTREE, accept_len 0, next_token -1 and a path of -1. */
+int fsd_verify_tree(const void *target_logits, const void *draft_logits,
+                    const int32_t *parent, const float *u_sample,
+                    int B, int N, int V, int max_depth, const fsd_opts *opts,
+                    int32_t *accept_len, int32_t *path, int32_t *next_token, float *divergence,
+                    int32_t *row_status, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Human-readable name of a host status code (static storage, never NULL). */
+const char *fsd_status_string(int status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int fsd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FSD_VERIFY_H */

@@ -1,0 +1,14 @@
+"""B200 (sm_100a) verification step of Fuzzy Speculative Decoding: Python binding of the C ABI."""
+
+from .binding import (  # noqa: F401
+    FsdOpts,
+    FsdError,
+    fsd_default_opts,
+    fsd_status_string,
+    fsd_verify_chain,
+    fsd_verify_tree,
+    fsd_version,
+    fsd_workspace_bytes,
+    library_path,
+    make_opts,
+)

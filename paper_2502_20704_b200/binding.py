@@ -1,0 +1,135 @@
+"""ctypes binding of libfsd_verify.so.
+
+The functions here carry the names and argument order of the C entry points and do
+argument marshalling only: tensors become device pointers, the options become the C
+struct.  There is no fallback: if the compiled library is missing, importing a
+function from it raises.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "lib", "libfsd_verify.so")
+
+DIVS = {"js": 0, "kl": 1, "tv": 2}
+MODES = {"fsd": 0, "sd": 1, "rfsd": 2}
+CMPS = {"lt": 0, "le": 1}
+SAMPLES = {"invcdf": 0, "greedy": 1}
+DTYPES = {"f32": 0, "bf16": 1}
+
+FSD_OK = 0
+FSD_ERR_NULL, FSD_ERR_SHAPE, FSD_ERR_ALIGN, FSD_ERR_ENUM = -1, -2, -3, -4
+FSD_ERR_WORKSPACE, FSD_ERR_UNSUPPORTED, FSD_ERR_CUDA = -5, -6, -7
+FSD_ROW_NONFINITE, FSD_ROW_TIMEOUT, FSD_ROW_BADTREE = 1, 2, 4
+
+
+class FsdOpts(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32),
+        ("divergence", C.c_int32),
+        ("mode", C.c_int32),
+        ("compare", C.c_int32),
+        ("sample", C.c_int32),
+        ("logit_dtype", C.c_int32),
+        ("threshold", C.c_float),
+    ]
+
+
+class FsdError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(f"fsd_verify failed: {fsd_status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2502_20704_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        lib = C.CDLL(_LIB_PATH)
+        vp, ip, fp = C.c_void_p, C.c_void_p, C.c_void_p
+        lib.fsd_default_opts.argtypes = [C.POINTER(FsdOpts)]
+        lib.fsd_default_opts.restype = None
+        lib.fsd_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts), C.POINTER(C.c_size_t)]
+        lib.fsd_workspace_bytes.restype = C.c_int
+        lib.fsd_verify_chain.argtypes = [vp, vp, ip, fp, fp, C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts),
+                                         ip, ip, fp, ip, vp, C.c_size_t, vp]
+        lib.fsd_verify_chain.restype = C.c_int
+        lib.fsd_verify_tree.argtypes = [vp, vp, ip, fp, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts),
+                                        ip, ip, ip, fp, ip, vp, C.c_size_t, vp]
+        lib.fsd_verify_tree.restype = C.c_int
+        lib.fsd_status_string.argtypes = [C.c_int]
+        lib.fsd_status_string.restype = C.c_char_p
+        lib.fsd_version.restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or raw integer) pointer of a tensor-like argument; None stays NULL."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def fsd_default_opts() -> FsdOpts:
+    o = FsdOpts()
+    _load().fsd_default_opts(C.byref(o))
+    return o
+
+
+def make_opts(div="js", mode="fsd", cmp="lt", sample="invcdf", dtype="bf16", T=0.0) -> FsdOpts:
+    o = fsd_default_opts()
+    o.divergence, o.mode, o.compare = DIVS[div], MODES[mode], CMPS[cmp]
+    o.sample, o.logit_dtype, o.threshold = SAMPLES[sample], DTYPES[dtype], float(T)
+    return o
+
+
+def fsd_status_string(status: int) -> str:
+    return _load().fsd_status_string(int(status)).decode()
+
+
+def fsd_version() -> int:
+    return _load().fsd_version()
+
+
+def fsd_workspace_bytes(B: int, positions: int, V: int, opts: FsdOpts) -> int:
+    out = C.c_size_t(0)
+    rc = _load().fsd_workspace_bytes(B, positions, V, C.byref(opts), C.byref(out))
+    if rc != FSD_OK:
+        raise FsdError(rc)
+    return out.value
+
+
+def fsd_verify_chain(target_logits, draft_logits, draft_tokens, u_accept, u_sample, B, gamma, V, opts,
+                     accept_len, next_token, divergence, row_status, workspace, workspace_bytes, stream=None) -> int:
+    """Same arguments as the C entry point; tensors (or integer addresses) are passed as pointers.
+    Returns the host status code (0 = OK)."""
+    return _load().fsd_verify_chain(_ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(u_accept),
+                                    _ptr(u_sample), B, gamma, V, C.byref(opts) if opts is not None else None,
+                                    _ptr(accept_len), _ptr(next_token), _ptr(divergence), _ptr(row_status),
+                                    _ptr(workspace), int(workspace_bytes), _ptr(stream))
+
+
+def fsd_verify_tree(target_logits, draft_logits, parent, u_sample, B, N, V, max_depth, opts,
+                    accept_len, path, next_token, divergence, row_status, workspace, workspace_bytes,
+                    stream=None) -> int:
+    return _load().fsd_verify_tree(_ptr(target_logits), _ptr(draft_logits), _ptr(parent), _ptr(u_sample),
+                                   B, N, V, max_depth, C.byref(opts) if opts is not None else None,
+                                   _ptr(accept_len), _ptr(path), _ptr(next_token), _ptr(divergence),
+                                   _ptr(row_status), _ptr(workspace), int(workspace_bytes), _ptr(stream))

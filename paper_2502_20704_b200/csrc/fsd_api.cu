@@ -1,0 +1,195 @@
+// C ABI of the verification library: argument checks, workspace layout, kernel launches.
+// See include/fsd_verify.h for the contract of every entry point.
+#include <climits>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "fsd_verify.h"
+#include "fsd_device.cuh"
+#include "fsd_finish.cuh"
+#include "fsd_pair_generic.cuh"
+
+namespace {
+
+using namespace fsd;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+struct Workspace {
+    int32_t* item_bits;
+    int32_t* item_status;
+    size_t bytes;
+};
+
+Workspace carve(void* base, int B, int G) {
+    Workspace w;
+    const size_t items = static_cast<size_t>(B) * G;
+    char* p = static_cast<char*>(base);
+    w.item_bits = reinterpret_cast<int32_t*>(p);
+    p += align_up(items * sizeof(int32_t));
+    w.item_status = reinterpret_cast<int32_t*>(p);
+    p += align_up(items * sizeof(int32_t));
+    w.bytes = static_cast<size_t>(p - static_cast<char*>(base));
+    return w;
+}
+
+int check_opts(const fsd_opts* o) {
+    if (o == nullptr) return FSD_ERR_NULL;
+    if (o->struct_size != sizeof(fsd_opts)) return FSD_ERR_ENUM;
+    if (o->divergence < FSD_DIV_JS || o->divergence > FSD_DIV_TV) return FSD_ERR_ENUM;
+    if (o->mode < FSD_MODE_FSD || o->mode > FSD_MODE_RFSD) return FSD_ERR_ENUM;
+    if (o->compare < FSD_CMP_LT || o->compare > FSD_CMP_LE) return FSD_ERR_ENUM;
+    if (o->sample < FSD_SAMPLE_INVCDF || o->sample > FSD_SAMPLE_GREEDY) return FSD_ERR_ENUM;
+    if (o->logit_dtype < FSD_F32 || o->logit_dtype > FSD_BF16) return FSD_ERR_ENUM;
+    if (o->threshold != o->threshold) return FSD_ERR_ENUM;   // NaN threshold
+    return FSD_OK;
+}
+
+int check_shape(int B, int G, int V) {
+    if (B < 1 || G < 1 || V < 1) return FSD_ERR_SHAPE;
+    if (static_cast<long long>(B) * (static_cast<long long>(G) + 1) > INT_MAX) return FSD_ERR_SHAPE;
+    return FSD_OK;
+}
+
+int finish_cluster_size(int V) {
+    // about 32 vocabulary entries per thread, at most the portable cluster size
+    int cs = 1;
+    while (cs < kMaxClusterSize && static_cast<long long>(cs) * kFinishThreads * 32 < V) cs <<= 1;
+    return cs;
+}
+
+template <int DT>
+int launch_all(const PairParams& pp, const FinishParams& fp, bool vec, cudaStream_t s) {
+    const int items = pp.B * pp.G;
+    if (vec) fsd_pair_generic_kernel<DT, true><<<items, 512, 0, s>>>(pp);
+    else     fsd_pair_generic_kernel<DT, false><<<items, 512, 0, s>>>(pp);
+    if (cudaGetLastError() != cudaSuccess) return FSD_ERR_CUDA;
+
+    const int cs = finish_cluster_size(fp.V);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(fp.B) * cs, 1, 1);
+    cfg.blockDim = dim3(kFinishThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, fsd_finish_kernel<DT>, fp) != cudaSuccess) return FSD_ERR_CUDA;
+    return FSD_OK;
+}
+
+int verify_common(const void* target, const void* draft, const int32_t* tokens, const float* u_accept,
+                  const float* u_sample, const int32_t* parent, int B, int G, int V, int max_depth,
+                  const fsd_opts* o, int32_t* accept_len, int32_t* path, int32_t* next_token,
+                  float* divergence, int32_t* row_status, void* workspace, size_t workspace_bytes,
+                  void* stream) {
+    const size_t es = o->logit_dtype == FSD_BF16 ? 2 : 4;
+    if (!aligned(target, es) || !aligned(draft, es) || !aligned(u_sample, 4) || !aligned(accept_len, 4) ||
+        !aligned(next_token, 4) || !aligned(divergence, 4) || !aligned(row_status, 4) ||
+        !aligned(tokens, 4) || !aligned(u_accept, 4) || !aligned(parent, 4) || !aligned(path, 4) ||
+        !aligned(workspace, kAlign))
+        return FSD_ERR_ALIGN;
+    Workspace ws = carve(workspace, B, G);
+    if (workspace_bytes < ws.bytes) return FSD_ERR_WORKSPACE;
+
+    PairParams pp;
+    pp.target = target; pp.draft = draft; pp.tokens = tokens; pp.u_accept = u_accept; pp.parent = parent;
+    pp.B = B; pp.G = G; pp.V = V;
+    pp.div = o->divergence; pp.mode = o->mode; pp.cmp = o->compare; pp.T = o->threshold;
+    pp.divergence = divergence; pp.item_bits = ws.item_bits; pp.item_status = ws.item_status;
+
+    FinishParams fp;
+    fp.target = target; fp.draft = draft; fp.parent = parent; fp.u_sample = u_sample;
+    fp.B = B; fp.G = G; fp.V = V;
+    fp.mode = o->mode; fp.sample = o->sample; fp.max_depth = max_depth;
+    fp.item_bits = ws.item_bits; fp.item_status = ws.item_status;
+    fp.accept_len = accept_len; fp.path = path; fp.next_token = next_token; fp.row_status = row_status;
+
+    const bool vec = (static_cast<size_t>(V) * es) % 16 == 0 && aligned(target, 16) && aligned(draft, 16);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, s) : launch_all<FSD_F32>(pp, fp, vec, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+void fsd_default_opts(fsd_opts* opts) {
+    if (opts == nullptr) return;
+    opts->struct_size = sizeof(fsd_opts);
+    opts->divergence = FSD_DIV_JS;
+    opts->mode = FSD_MODE_FSD;
+    opts->compare = FSD_CMP_LT;
+    opts->sample = FSD_SAMPLE_INVCDF;
+    opts->logit_dtype = FSD_BF16;
+    opts->threshold = 0.0f;
+}
+
+int fsd_workspace_bytes(int B, int positions, int V, const fsd_opts* opts, size_t* bytes_out) {
+    if (bytes_out == nullptr) return FSD_ERR_NULL;
+    int rc = check_opts(opts);
+    if (rc != FSD_OK) return rc;
+    rc = check_shape(B, positions, V);
+    if (rc != FSD_OK) return rc;
+    *bytes_out = carve(nullptr, B, positions).bytes;
+    return FSD_OK;
+}
+
+int fsd_verify_chain(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                     const float* u_accept, const float* u_sample, int B, int gamma, int V,
+                     const fsd_opts* opts, int32_t* accept_len, int32_t* next_token, float* divergence,
+                     int32_t* row_status, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_opts(opts);
+    if (rc != FSD_OK) return rc;
+    if (!target_logits || !draft_logits || !u_sample || !accept_len || !next_token || !divergence ||
+        !row_status || !workspace)
+        return FSD_ERR_NULL;
+    if (opts->mode != FSD_MODE_FSD && (!draft_tokens || !u_accept)) return FSD_ERR_NULL;
+    rc = check_shape(B, gamma, V);
+    if (rc != FSD_OK) return rc;
+    return verify_common(target_logits, draft_logits, draft_tokens, u_accept, u_sample, nullptr, B, gamma, V, 0,
+                         opts, accept_len, nullptr, next_token, divergence, row_status, workspace,
+                         workspace_bytes, stream);
+}
+
+int fsd_verify_tree(const void* target_logits, const void* draft_logits, const int32_t* parent,
+                    const float* u_sample, int B, int N, int V, int max_depth, const fsd_opts* opts,
+                    int32_t* accept_len, int32_t* path, int32_t* next_token, float* divergence,
+                    int32_t* row_status, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_opts(opts);
+    if (rc != FSD_OK) return rc;
+    if (!target_logits || !draft_logits || !parent || !u_sample || !accept_len || !path || !next_token ||
+        !divergence || !row_status || !workspace)
+        return FSD_ERR_NULL;
+    if (opts->mode != FSD_MODE_FSD) return FSD_ERR_UNSUPPORTED;
+    rc = check_shape(B, N, V);
+    if (rc != FSD_OK) return rc;
+    if (max_depth < 1 || N > kMaxTreeNodes) return FSD_ERR_SHAPE;
+    return verify_common(target_logits, draft_logits, nullptr, nullptr, u_sample, parent, B, N, V, max_depth,
+                         opts, accept_len, path, next_token, divergence, row_status, workspace,
+                         workspace_bytes, stream);
+}
+
+const char* fsd_status_string(int status) {
+    switch (status) {
+        case FSD_OK: return "FSD_OK";
+        case FSD_ERR_NULL: return "FSD_ERR_NULL: a required pointer is NULL";
+        case FSD_ERR_SHAPE: return "FSD_ERR_SHAPE: a dimension is out of range";
+        case FSD_ERR_ALIGN: return "FSD_ERR_ALIGN: a pointer is misaligned";
+        case FSD_ERR_ENUM: return "FSD_ERR_ENUM: an option is out of range";
+        case FSD_ERR_WORKSPACE: return "FSD_ERR_WORKSPACE: workspace too small";
+        case FSD_ERR_UNSUPPORTED: return "FSD_ERR_UNSUPPORTED: combination not defined";
+        case FSD_ERR_CUDA: return "FSD_ERR_CUDA: the CUDA runtime refused a launch";
+        default: return "unknown fsd status";
+    }
+}
+
+int fsd_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,203 @@
+"""GPU-vs-oracle parity through the C ABI (see tests/parity.py for the comparison rules)."""
+
+import numpy as np
+import pytest
+
+import fsd_inputs as gi
+from oracle import fsd_oracle as orc
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(c, **kw):
+    return parity.check_chain(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, **kw)
+
+
+# --------------------------------------------------------------------------- #
+# the five named workloads
+# --------------------------------------------------------------------------- #
+def test_config1_all_divergences_thresholds_and_compare_ops():
+    c = gi.make_config("c1")
+    for div in ("js", "kl", "tv"):
+        for T in gi.CONFIGS["c1"].thresholds:
+            for cmp in ("lt", "le"):
+                r = _check(c, div=div, T=T, cmp=cmp)
+                assert r["max_err"] <= 1e-5
+
+
+def test_config2_fsd_and_sd_threshold_sweep():
+    c = gi.make_config("c2")
+    lens = []
+    for T in gi.CONFIGS["c2"].thresholds:
+        r = _check(c, mode="fsd", T=T)
+        lens.append(r["accept_len"])
+        assert r["max_err"] <= 1e-4
+    assert all((b >= a).all() for a, b in zip(lens, lens[1:]))       # larger T never accepts less
+    assert lens[0].max() == 0 and lens[-1].min() == c.gamma
+    _check(c, mode="sd", T=0.0)
+    for T in (0.0, 2.0 / 7):
+        _check(c, mode="rfsd", T=T)
+    for sample in ("greedy",):
+        _check(c, mode="fsd", T=1.0 / 7, sample=sample)
+        _check(c, mode="sd", sample=sample)
+
+
+def test_config3_zipf_with_disjoint_drafts():
+    c = gi.make_config("c3")
+    for T in gi.CONFIGS["c3"].thresholds:
+        r = _check(c, T=T)
+        assert r["max_err"] <= 1e-4
+    assert c.disjoint.any()
+    r = _check(c, div="kl", T=0.3)
+    r = _check(c, div="tv", T=0.3)
+
+
+def test_config4_headline_shape():
+    c = gi.make_config("c4")
+    r = _check(c, T=0.2)
+    assert r["max_err"] <= 1e-4
+    assert len(set(r["accept_len"].tolist())) > 2                    # the workload is not degenerate
+    _check(c, T=0.2, cmp="le")
+
+
+def test_config5_tree():
+    c = gi.make_config("c5")
+    tol = 1e-4
+    for T in gi.CONFIGS["c5"].thresholds:
+        g = parity.run_tree_gpu(c.target, c.draft, c.parent, c.u_sample, c.max_depth, c.dtype, T=T)
+        o = orc.verify_tree(c.target, c.draft, c.parent, c.u_sample, c.max_depth, dtype=c.dtype, T=T,
+                            band=parity.SAMPLE_BAND)
+        parity.compare_divergence(g.divergence, o.divergence, tol)
+        in_band = np.abs(o.divergence - float(np.float32(T))) < parity.D_BAND
+        for b in range(c.B):
+            if in_band[b].any():
+                forced = np.full((1, c.N), -1, dtype=np.int8)
+                forced[0, in_band[b]] = (g.divergence[b, in_band[b]] < np.float32(T)).astype(np.int8)
+                ob = orc.verify_tree(c.target[b:b + 1], c.draft[b:b + 1], c.parent[b:b + 1], c.u_sample[b:b + 1],
+                                     c.max_depth, dtype=c.dtype, T=T, band=parity.SAMPLE_BAND, forced=forced)
+                n_o, p_o, t_o = ob.accept_len[0], ob.path[0], ob.next_token[0]
+            else:
+                n_o, p_o, t_o = o.accept_len[b], o.path[b], o.next_token[b]
+            assert g.accept_len[b] == n_o and np.array_equal(g.path[b], p_o) and g.next_token[b] == t_o
+        assert np.array_equal(g.row_status, o.row_status)
+
+
+# --------------------------------------------------------------------------- #
+# small, odd and degenerate shapes
+# --------------------------------------------------------------------------- #
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 2, 7, 8, 33, 1000, 4099, 20000])
+def test_odd_vocabulary_sizes(dtype, V):
+    c = gi.make_chain(3, 2, V, dtype=dtype, recipe="spike", sigma=(0.3, 1.0), workload_id=100 + V)
+    for div in ("js", "kl", "tv"):
+        _check(c, div=div, T=0.1)
+    _check(c, mode="sd")
+    _check(c, mode="rfsd", T=0.05)
+
+
+def test_gamma_one_and_long_chains():
+    for gamma in (1, 20, 70):
+        c = gi.make_chain(2, gamma, 512, dtype="bf16", recipe="zipf", sigma=(0.2, 0.6), sigma_mode="uniform",
+                          workload_id=200 + gamma)
+        _check(c, T=0.05)
+        _check(c, T=10.0)
+
+
+def test_identical_rows_and_threshold_zero():
+    c = gi.make_chain(4, 3, 4096, dtype="bf16", recipe="spike", sigma=(0.5,), workload_id=300)
+    c.draft[0, 0] = c.target[0, 0]
+    c.draft[0, 1] = c.target[0, 1]
+    c.draft[2, 0] = c.target[2, 0]
+    r = _check(c, T=0.0, cmp="le")
+    assert r["accept_len"].tolist() == [2, 0, 1, 0]
+    assert r["gpu"].divergence[0, 0] == 0.0 and r["gpu"].divergence[2, 0] == 0.0
+    r = _check(c, T=0.0, cmp="lt")
+    assert (r["accept_len"] == 0).all()
+    for div in ("kl", "tv"):
+        r = _check(c, T=0.0, cmp="le", div=div)
+        assert r["gpu"].divergence[0, 1] == 0.0
+
+
+def test_masked_logits_and_disjoint_supports():
+    c = gi.make_chain(3, 2, 1024, dtype="f32", recipe="spike", sigma=(0.5,), workload_id=301)
+    c.target[0, 0, 512:] = -np.inf
+    c.draft[0, 0, :512] = -np.inf                 # disjoint: JS = ln 2, TV = 1, KL = inf
+    c.target[1, 1, ::3] = -np.inf                 # masked target entries only
+    c.draft[2, 0, 5::7] = -np.inf                 # masked draft entries: KL = inf
+    for div in ("js", "kl", "tv"):
+        r = _check(c, div=div, T=0.7)
+    r = _check(c, div="js", T=0.7)
+    assert abs(r["gpu"].divergence[0, 0] - np.log(2.0)) < 1e-6
+    r = _check(c, div="kl", T=100.0)
+    assert np.isposinf(r["gpu"].divergence[0, 0]) and np.isposinf(r["gpu"].divergence[2, 0])
+    _check(c, mode="sd")
+
+
+def test_nonfinite_rows_are_flagged_not_propagated():
+    c = gi.make_chain(4, 3, 2048, dtype="f32", recipe="spike", sigma=(0.5,), workload_id=302)
+    c.draft[0, 1, 17] = np.nan
+    c.target[1, 0, 3] = np.inf
+    c.target[2, 3, :] = -np.inf                   # the bonus row of row 2 has no finite entry
+    r = _check(c, T=100.0)
+    assert r["gpu"].row_status.tolist() == [1, 1, 1, 0]
+    assert r["accept_len"].tolist() == [1, 0, 3, 3]
+    assert r["gpu"].next_token[1] == -1 and r["gpu"].next_token[2] == -1
+    _check(c, mode="sd")
+
+
+def test_uniform_extremes_for_sampling():
+    c = gi.make_chain(6, 2, 5000, dtype="bf16", recipe="zipf", sigma=(0.5,), workload_id=303)
+    c.u_sample[:] = np.array([0.0, np.nextafter(np.float32(1), np.float32(0)), 0.5, 1e-7, 0.999, 0.25], np.float32)
+    _check(c, T=0.0)
+    _check(c, T=10.0)
+    c.u_accept[:] = 0.0
+    _check(c, mode="sd")
+
+
+def test_fsd_outputs_do_not_depend_on_tokens_or_accept_uniforms():
+    c = gi.make_chain(4, 4, 3000, dtype="bf16", recipe="spike", sigma=(0.2, 1.5), sigma_mode="uniform", workload_id=304)
+    a = parity.run_chain_gpu(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, T=0.1)
+    b = parity.run_chain_gpu(c.target, c.draft, None, None, c.u_sample, c.dtype, T=0.1)
+    assert np.array_equal(a.accept_len, b.accept_len) and np.array_equal(a.next_token, b.next_token)
+    assert np.array_equal(a.divergence, b.divergence)
+    # bit-reproducible from run to run
+    a2 = parity.run_chain_gpu(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, T=0.1)
+    assert np.array_equal(a.divergence, a2.divergence) and np.array_equal(a.next_token, a2.next_token)
+
+
+def test_out_of_range_draft_token_is_rejected_in_sd_mode():
+    c = gi.make_chain(2, 3, 512, dtype="f32", recipe="spike", sigma=(0.1,), workload_id=305)
+    c.draft_tokens[0, 1] = 512
+    c.draft_tokens[1, 0] = -1
+    c.u_accept[:] = 0.0
+    r = _check(c, mode="sd")
+    assert r["accept_len"].tolist() == [1, 0]
+
+
+# --------------------------------------------------------------------------- #
+# trees
+# --------------------------------------------------------------------------- #
+def test_chain_shaped_tree_matches_chain_call():
+    B, N, V = 3, 5, 4096
+    parent = np.tile(np.arange(-1, N - 1, dtype=np.int32), (B, 1))
+    t = gi.make_tree(B, N, V, dtype="bf16", sigma=0.6, workload_id=400, parent=parent)
+    for T in (0.02, 0.045, 0.3):
+        g = parity.run_tree_gpu(t.target, t.draft, t.parent, t.u_sample, N, t.dtype, T=T)
+        c = parity.run_chain_gpu(t.target, t.draft, None, None, t.u_sample, t.dtype, T=T)
+        assert np.array_equal(g.accept_len, c.accept_len) and np.array_equal(g.next_token, c.next_token)
+        assert np.array_equal(g.divergence, c.divergence)
+
+
+def test_tree_max_depth_and_bad_parent():
+    t = gi.make_tree(3, 12, 2048, dtype="f32", sigma=0.3, max_depth=5, workload_id=401)
+    t.parent[1, 4] = 4                           # a node naming itself as parent
+    for depth in (1, 2, 5):
+        g = parity.run_tree_gpu(t.target, t.draft, t.parent, t.u_sample, depth, t.dtype, T=5.0)
+        o = orc.verify_tree(t.target, t.draft, t.parent, t.u_sample, depth, dtype=t.dtype, T=5.0,
+                            band=parity.SAMPLE_BAND)
+        assert np.array_equal(g.accept_len, o.accept_len) and np.array_equal(g.path, o.path)
+        assert np.array_equal(g.next_token, o.next_token) and np.array_equal(g.row_status, o.row_status)
+        assert g.row_status[1] & 4 and g.accept_len[1] == 0 and g.next_token[1] == -1
+        assert g.accept_len.max() <= depth
+        parity.compare_divergence(g.divergence, o.divergence, 1e-5)
