@@ -141,6 +141,20 @@ int fsd_verify_tree(const void *target_logits, const void *draft_logits,
                     int32_t *accept_len, int32_t *path, int32_t *next_token, float *divergence,
                     int32_t *row_status, void *workspace, size_t workspace_bytes, void *stream);
 
+/* Chain verification with HOST buffers (same computation as fsd_verify_chain).
+ * Every h_* pointer is a HOST pointer (pinned memory makes the copies faster; pageable works).
+ * The call copies the inputs into `staging` (device scratch, 256-byte aligned, at least
+ * fsd_host_staging_bytes() bytes, owned by the caller), runs fsd_verify_chain on them on
+ * `stream`, copies the four outputs back and synchronises the stream before it returns, so the
+ * host outputs are valid on return.  h_draft_tokens / h_u_accept may be NULL in FSD mode.
+ * Errors as fsd_verify_chain; a failed copy gives FSD_ERR_CUDA. */
+int fsd_host_staging_bytes(int B, int gamma, int V, const fsd_opts *opts, size_t *bytes_out);
+int fsd_verify_chain_host(const void *h_target_logits, const void *h_draft_logits,
+                          const int32_t *h_draft_tokens, const float *h_u_accept, const float *h_u_sample,
+                          int B, int gamma, int V, const fsd_opts *opts,
+                          int32_t *h_accept_len, int32_t *h_next_token, float *h_divergence,
+                          int32_t *h_row_status, void *staging, size_t staging_bytes, void *stream);
+
 /* Human-readable name of a host status code (static storage, never NULL). */
 const char *fsd_status_string(int status);
 

@@ -4,8 +4,10 @@ from .binding import (  # noqa: F401
     FsdOpts,
     FsdError,
     fsd_default_opts,
+    fsd_host_staging_bytes,
     fsd_status_string,
     fsd_verify_chain,
+    fsd_verify_chain_host,
     fsd_verify_tree,
     fsd_version,
     fsd_workspace_bytes,

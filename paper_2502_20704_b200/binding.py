@@ -71,6 +71,11 @@ def _load():
         lib.fsd_verify_tree.argtypes = [vp, vp, ip, fp, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts),
                                         ip, ip, ip, fp, ip, vp, C.c_size_t, vp]
         lib.fsd_verify_tree.restype = C.c_int
+        lib.fsd_host_staging_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts), C.POINTER(C.c_size_t)]
+        lib.fsd_host_staging_bytes.restype = C.c_int
+        lib.fsd_verify_chain_host.argtypes = [vp, vp, ip, fp, fp, C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts),
+                                              ip, ip, fp, ip, vp, C.c_size_t, vp]
+        lib.fsd_verify_chain_host.restype = C.c_int
         lib.fsd_status_string.argtypes = [C.c_int]
         lib.fsd_status_string.restype = C.c_char_p
         lib.fsd_version.restype = C.c_int
@@ -133,3 +138,22 @@ def fsd_verify_tree(target_logits, draft_logits, parent, u_sample, B, N, V, max_
                                    B, N, V, max_depth, C.byref(opts) if opts is not None else None,
                                    _ptr(accept_len), _ptr(path), _ptr(next_token), _ptr(divergence),
                                    _ptr(row_status), _ptr(workspace), int(workspace_bytes), _ptr(stream))
+
+
+def fsd_host_staging_bytes(B: int, gamma: int, V: int, opts: FsdOpts) -> int:
+    out = C.c_size_t(0)
+    rc = _load().fsd_host_staging_bytes(B, gamma, V, C.byref(opts), C.byref(out))
+    if rc != FSD_OK:
+        raise FsdError(rc)
+    return out.value
+
+
+def fsd_verify_chain_host(h_target_logits, h_draft_logits, h_draft_tokens, h_u_accept, h_u_sample, B, gamma, V,
+                          opts, h_accept_len, h_next_token, h_divergence, h_row_status, staging, staging_bytes,
+                          stream=None) -> int:
+    """Host-buffer variant: the h_* arguments are CPU tensors (ideally pinned), `staging` a device tensor."""
+    return _load().fsd_verify_chain_host(_ptr(h_target_logits), _ptr(h_draft_logits), _ptr(h_draft_tokens),
+                                         _ptr(h_u_accept), _ptr(h_u_sample), B, gamma, V,
+                                         C.byref(opts) if opts is not None else None, _ptr(h_accept_len),
+                                         _ptr(h_next_token), _ptr(h_divergence), _ptr(h_row_status),
+                                         _ptr(staging), int(staging_bytes), _ptr(stream))

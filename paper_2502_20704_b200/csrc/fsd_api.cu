@@ -116,6 +116,29 @@ int verify_common(const void* target, const void* draft, const int32_t* tokens, 
     return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, s) : launch_all<FSD_F32>(pp, fp, vec, s);
 }
 
+struct HostStaging {
+    char *target, *draft, *tokens, *u_accept, *u_sample, *accept_len, *next_token, *divergence, *row_status, *ws;
+    size_t n_target, n_draft, n_items4, n_rows4, n_ws, bytes;
+};
+
+HostStaging carve_staging(void* base, int B, int G, int V, size_t es) {
+    HostStaging h;
+    h.n_target = static_cast<size_t>(B) * (G + 1) * V * es;
+    h.n_draft = static_cast<size_t>(B) * G * V * es;
+    h.n_items4 = static_cast<size_t>(B) * G * 4;
+    h.n_rows4 = static_cast<size_t>(B) * 4;
+    h.n_ws = carve(nullptr, B, G).bytes;
+    char* p = static_cast<char*>(base);
+    auto take = [&](size_t n) { char* q = p; p += align_up(n); return q; };
+    h.target = take(h.n_target); h.draft = take(h.n_draft);
+    h.tokens = take(h.n_items4); h.u_accept = take(h.n_items4); h.u_sample = take(h.n_rows4);
+    h.accept_len = take(h.n_rows4); h.next_token = take(h.n_rows4);
+    h.divergence = take(h.n_items4); h.row_status = take(h.n_rows4);
+    h.ws = take(h.n_ws);
+    h.bytes = static_cast<size_t>(p - static_cast<char*>(base));
+    return h;
+}
+
 }  // namespace
 
 extern "C" {
@@ -174,6 +197,55 @@ int fsd_verify_tree(const void* target_logits, const void* draft_logits, const i
     return verify_common(target_logits, draft_logits, nullptr, nullptr, u_sample, parent, B, N, V, max_depth,
                          opts, accept_len, path, next_token, divergence, row_status, workspace,
                          workspace_bytes, stream);
+}
+
+int fsd_host_staging_bytes(int B, int gamma, int V, const fsd_opts* opts, size_t* bytes_out) {
+    if (bytes_out == nullptr) return FSD_ERR_NULL;
+    int rc = check_opts(opts);
+    if (rc != FSD_OK) return rc;
+    rc = check_shape(B, gamma, V);
+    if (rc != FSD_OK) return rc;
+    *bytes_out = carve_staging(nullptr, B, gamma, V, opts->logit_dtype == FSD_BF16 ? 2 : 4).bytes;
+    return FSD_OK;
+}
+
+int fsd_verify_chain_host(const void* h_target_logits, const void* h_draft_logits, const int32_t* h_draft_tokens,
+                          const float* h_u_accept, const float* h_u_sample, int B, int gamma, int V,
+                          const fsd_opts* opts, int32_t* h_accept_len, int32_t* h_next_token,
+                          float* h_divergence, int32_t* h_row_status, void* staging, size_t staging_bytes,
+                          void* stream) {
+    int rc = check_opts(opts);
+    if (rc != FSD_OK) return rc;
+    if (!h_target_logits || !h_draft_logits || !h_u_sample || !h_accept_len || !h_next_token || !h_divergence ||
+        !h_row_status || !staging)
+        return FSD_ERR_NULL;
+    if (opts->mode != FSD_MODE_FSD && (!h_draft_tokens || !h_u_accept)) return FSD_ERR_NULL;
+    rc = check_shape(B, gamma, V);
+    if (rc != FSD_OK) return rc;
+    if (!aligned(staging, kAlign)) return FSD_ERR_ALIGN;
+    HostStaging h = carve_staging(staging, B, gamma, V, opts->logit_dtype == FSD_BF16 ? 2 : 4);
+    if (staging_bytes < h.bytes) return FSD_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    bool ok = true;
+    ok = ok && cudaMemcpyAsync(h.target, h_target_logits, h.n_target, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(h.draft, h_draft_logits, h.n_draft, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (h_draft_tokens) ok = ok && cudaMemcpyAsync(h.tokens, h_draft_tokens, h.n_items4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (h_u_accept) ok = ok && cudaMemcpyAsync(h.u_accept, h_u_accept, h.n_items4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(h.u_sample, h_u_sample, h.n_rows4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) return FSD_ERR_CUDA;
+    rc = fsd_verify_chain(h.target, h.draft, h_draft_tokens ? reinterpret_cast<int32_t*>(h.tokens) : nullptr,
+                          h_u_accept ? reinterpret_cast<float*>(h.u_accept) : nullptr,
+                          reinterpret_cast<float*>(h.u_sample), B, gamma, V, opts,
+                          reinterpret_cast<int32_t*>(h.accept_len), reinterpret_cast<int32_t*>(h.next_token),
+                          reinterpret_cast<float*>(h.divergence), reinterpret_cast<int32_t*>(h.row_status),
+                          h.ws, h.n_ws, stream);
+    if (rc != FSD_OK) return rc;
+    ok = ok && cudaMemcpyAsync(h_accept_len, h.accept_len, h.n_rows4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(h_next_token, h.next_token, h.n_rows4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(h_divergence, h.divergence, h.n_items4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(h_row_status, h.row_status, h.n_rows4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
+    return ok ? FSD_OK : FSD_ERR_CUDA;
 }
 
 const char* fsd_status_string(int status) {
