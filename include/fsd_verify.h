@@ -75,6 +75,7 @@ extern "C" {
 #define FSD_ERR_WORKSPACE   -5  /* workspace_bytes is smaller than fsd_workspace_bytes() reports */
 #define FSD_ERR_UNSUPPORTED -6  /* combination not defined (SD / rFSD on a tree) */
 #define FSD_ERR_CUDA        -7  /* the CUDA runtime refused a launch or a copy */
+#define FSD_ERR_TOO_LARGE   -8  /* B * gamma exceeds what the built-in scratch of fsd_verify_chain_static holds */
 
 /* row_status bit flags (device-side conditions) */
 #define FSD_ROW_NONFINITE 1  /* some logit row read for this batch row was not a valid distribution */
@@ -154,6 +155,38 @@ int fsd_verify_chain_host(const void *h_target_logits, const void *h_draft_logit
                           int B, int gamma, int V, const fsd_opts *opts,
                           int32_t *h_accept_len, int32_t *h_next_token, float *h_divergence,
                           int32_t *h_row_status, void *staging, size_t staging_bytes, void *stream);
+
+/* Chain verification for callers that cannot provide scratch memory.
+ * (The paper has no counterpart to this entry point; it exists for integration only.)
+ *
+ * Some hosts of this library are not allowed to allocate device memory at the point where they
+ * verify: a decoding loop whose memory pool was sized and frozen at start-up, a plugin that runs
+ * inside another framework's allocator and must not go around it, a serving process whose whole
+ * device budget is already handed out.  Such a caller has no buffer to pass as `workspace` and
+ * cannot call cudaMalloc to get one.  This variant computes exactly what fsd_verify_chain
+ * computes, with the same kernels, but keeps the per-position accept bits and status words in a
+ * fixed array that is part of the library's device image, so the caller passes only inputs and
+ * outputs.  It calls no cudaMalloc, cudaFree or any other allocating routine.
+ *
+ * Limits and rules
+ *   - B * gamma must not exceed FSD_STATIC_MAX_POSITIONS; larger calls are refused with
+ *     FSD_ERR_TOO_LARGE and nothing is launched.  The array (FSD_STATIC_SCRATCH_BYTES, 64 KiB)
+ *     is resident on every GPU that loads the library until the process exits.
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     Nothing in it has to start at zero: every word a call reads was written earlier by the
+ *     same call.  Two calls that overlap on the GPU (different streams, no ordering between
+ *     them) race on it and give wrong results; order them, or use fsd_verify_chain with
+ *     separate workspaces.
+ * Arguments, outputs and the other error codes are those of fsd_verify_chain. */
+#define FSD_STATIC_SCRATCH_BYTES 65536
+#define FSD_STATIC_MAX_POSITIONS 8128
+int fsd_verify_chain_static(const void *target_logits, const void *draft_logits,
+                            const int32_t *draft_tokens, const float *u_accept, const float *u_sample,
+                            int B, int gamma, int V, const fsd_opts *opts,
+                            int32_t *accept_len, int32_t *next_token, float *divergence,
+                            int32_t *row_status, void *stream);
 
 /* Human-readable name of a host status code (static storage, never NULL). */
 const char *fsd_status_string(int status);

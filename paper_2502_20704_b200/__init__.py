@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     fsd_status_string,
     fsd_verify_chain,
     fsd_verify_chain_host,
+    fsd_verify_chain_static,
     fsd_verify_tree,
     fsd_version,
     fsd_workspace_bytes,

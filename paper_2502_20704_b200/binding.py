@@ -23,7 +23,8 @@ DTYPES = {"f32": 0, "bf16": 1}
 
 FSD_OK = 0
 FSD_ERR_NULL, FSD_ERR_SHAPE, FSD_ERR_ALIGN, FSD_ERR_ENUM = -1, -2, -3, -4
-FSD_ERR_WORKSPACE, FSD_ERR_UNSUPPORTED, FSD_ERR_CUDA = -5, -6, -7
+FSD_ERR_WORKSPACE, FSD_ERR_UNSUPPORTED, FSD_ERR_CUDA, FSD_ERR_TOO_LARGE = -5, -6, -7, -8
+FSD_STATIC_MAX_POSITIONS = 8128
 FSD_ROW_NONFINITE, FSD_ROW_TIMEOUT, FSD_ROW_BADTREE = 1, 2, 4
 
 
@@ -76,6 +77,9 @@ def _load():
         lib.fsd_verify_chain_host.argtypes = [vp, vp, ip, fp, fp, C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts),
                                               ip, ip, fp, ip, vp, C.c_size_t, vp]
         lib.fsd_verify_chain_host.restype = C.c_int
+        lib.fsd_verify_chain_static.argtypes = [vp, vp, ip, fp, fp, C.c_int, C.c_int, C.c_int, C.POINTER(FsdOpts),
+                                                ip, ip, fp, ip, vp]
+        lib.fsd_verify_chain_static.restype = C.c_int
         lib.fsd_status_string.argtypes = [C.c_int]
         lib.fsd_status_string.restype = C.c_char_p
         lib.fsd_version.restype = C.c_int
@@ -157,3 +161,13 @@ def fsd_verify_chain_host(h_target_logits, h_draft_logits, h_draft_tokens, h_u_a
                                          C.byref(opts) if opts is not None else None, _ptr(h_accept_len),
                                          _ptr(h_next_token), _ptr(h_divergence), _ptr(h_row_status),
                                          _ptr(staging), int(staging_bytes), _ptr(stream))
+
+
+def fsd_verify_chain_static(target_logits, draft_logits, draft_tokens, u_accept, u_sample, B, gamma, V, opts,
+                            accept_len, next_token, divergence, row_status, stream=None) -> int:
+    """fsd_verify_chain for callers that may not allocate device memory: no workspace argument,
+    the scratch lives inside the library (B * gamma <= FSD_STATIC_MAX_POSITIONS)."""
+    return _load().fsd_verify_chain_static(_ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens),
+                                           _ptr(u_accept), _ptr(u_sample), B, gamma, V,
+                                           C.byref(opts) if opts is not None else None, _ptr(accept_len),
+                                           _ptr(next_token), _ptr(divergence), _ptr(row_status), _ptr(stream))

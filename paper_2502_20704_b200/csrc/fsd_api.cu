@@ -3,6 +3,7 @@
 #include <climits>
 #include <cstdint>
 #include <cuda_runtime.h>
+#include <mutex>
 
 #include "fsd_verify.h"
 #include "fsd_device.cuh"
@@ -139,6 +140,28 @@ HostStaging carve_staging(void* base, int B, int G, int V, size_t es) {
     return h;
 }
 
+// Built-in scratch of fsd_verify_chain_static.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the kernels get the device address that call returns.
+static __device__ __align__(256) unsigned char g_static_scratch[FSD_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device (looked up once per device).
+int static_scratch(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FSD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return FSD_ERR_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return FSD_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -248,6 +271,28 @@ int fsd_verify_chain_host(const void* h_target_logits, const void* h_draft_logit
     return ok ? FSD_OK : FSD_ERR_CUDA;
 }
 
+int fsd_verify_chain_static(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                            const float* u_accept, const float* u_sample, int B, int gamma, int V,
+                            const fsd_opts* opts, int32_t* accept_len, int32_t* next_token, float* divergence,
+                            int32_t* row_status, void* stream) {
+    int rc = check_opts(opts);
+    if (rc != FSD_OK) return rc;
+    if (!target_logits || !draft_logits || !u_sample || !accept_len || !next_token || !divergence || !row_status)
+        return FSD_ERR_NULL;
+    if (opts->mode != FSD_MODE_FSD && (!draft_tokens || !u_accept)) return FSD_ERR_NULL;
+    rc = check_shape(B, gamma, V);
+    if (rc != FSD_OK) return rc;
+    if (static_cast<long long>(B) * gamma > FSD_STATIC_MAX_POSITIONS ||
+        carve(nullptr, B, gamma).bytes > FSD_STATIC_SCRATCH_BYTES)
+        return FSD_ERR_TOO_LARGE;
+    void* scratch = nullptr;
+    rc = static_scratch(&scratch);
+    if (rc != FSD_OK) return rc;
+    return verify_common(target_logits, draft_logits, draft_tokens, u_accept, u_sample, nullptr, B, gamma, V, 0,
+                         opts, accept_len, nullptr, next_token, divergence, row_status, scratch,
+                         FSD_STATIC_SCRATCH_BYTES, stream);
+}
+
 const char* fsd_status_string(int status) {
     switch (status) {
         case FSD_OK: return "FSD_OK";
@@ -258,6 +303,7 @@ const char* fsd_status_string(int status) {
         case FSD_ERR_WORKSPACE: return "FSD_ERR_WORKSPACE: workspace too small";
         case FSD_ERR_UNSUPPORTED: return "FSD_ERR_UNSUPPORTED: combination not defined";
         case FSD_ERR_CUDA: return "FSD_ERR_CUDA: the CUDA runtime refused a launch";
+        case FSD_ERR_TOO_LARGE: return "FSD_ERR_TOO_LARGE: B * gamma exceeds FSD_STATIC_MAX_POSITIONS";
         default: return "unknown fsd status";
     }
 }
