@@ -9,6 +9,7 @@
 #include "fsd_device.cuh"
 #include "fsd_finish.cuh"
 #include "fsd_pair_generic.cuh"
+#include "fsd_pair_stream.cuh"
 
 namespace {
 
@@ -21,6 +22,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 struct Workspace {
     int32_t* item_bits;
     int32_t* item_status;
+    int* flags;                // [0] = a bounded device-side wait ran out
     size_t bytes;
 };
 
@@ -32,6 +34,8 @@ Workspace carve(void* base, int B, int G) {
     p += align_up(items * sizeof(int32_t));
     w.item_status = reinterpret_cast<int32_t*>(p);
     p += align_up(items * sizeof(int32_t));
+    w.flags = reinterpret_cast<int*>(p);
+    p += kAlign;
     w.bytes = static_cast<size_t>(p - static_cast<char*>(base));
     return w;
 }
@@ -61,12 +65,79 @@ int finish_cluster_size(int V) {
     return cs;
 }
 
+// ---- streaming kernel launch -----------------------------------------------------------
+constexpr int kMaxDev = 64;
+
+template <int DT, int DIV>
+int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
+    static int max_clusters[kMaxDev][4] = {};       // per device, per log2(C); 0 = not yet queried
+    static std::mutex mu;
+    auto kernel = fsd_pair_stream_kernel<DT, DIV>;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return FSD_ERR_CUDA;
+    int lc = 0;
+    while ((1 << lc) < C) ++lc;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.dynamicSmemBytes = kStreamSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int nclus;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (max_clusters[dev][lc] == 0) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+                return FSD_ERR_CUDA;
+            cfg.gridDim = dim3(C, 1, 1);
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) return FSD_ERR_CUDA;
+            max_clusters[dev][lc] = n;
+        }
+        nclus = max_clusters[dev][lc];
+    }
+    if (nclus > sp.n_items) nclus = sp.n_items;
+    cfg.gridDim = dim3(static_cast<unsigned>(nclus) * C, 1, 1);
+    if (cudaLaunchKernelEx(&cfg, kernel, sp) != cudaSuccess) return FSD_ERR_CUDA;
+    return FSD_OK;
+}
+
+// Cluster size for the streaming kernel: the smallest power of two whose per-CTA slice fits
+// on chip; 0 if the shape is not eligible (the generic kernel takes it).
+int stream_cluster_size(int nvec_row, bool vec) {
+    if (!vec || nvec_row < 64) return 0;
+    for (int C = 1; C <= kMaxClusterSize; C <<= 1)
+        if ((nvec_row + C - 1) / C <= kMaxVecPerCta) return C;
+    return 0;
+}
+
 template <int DT>
-int launch_all(const PairParams& pp, const FinishParams& fp, bool vec, cudaStream_t s) {
+int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, cudaStream_t s) {
     const int items = pp.B * pp.G;
-    if (vec) fsd_pair_generic_kernel<DT, true><<<items, 512, 0, s>>>(pp);
-    else     fsd_pair_generic_kernel<DT, false><<<items, 512, 0, s>>>(pp);
-    if (cudaGetLastError() != cudaSuccess) return FSD_ERR_CUDA;
+    const int nvec_row = pp.V / Logit<DT>::kPerVec;
+    const int C = stream_cluster_size(nvec_row, vec);
+    if (C > 0) {
+        StreamParams sp;
+        sp.pp = pp; sp.nvec_row = nvec_row; sp.n_items = items; sp.timeout_flag = flags;
+        int rc;
+        if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, C, s);
+        else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, C, s);
+        else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, C, s);
+        if (rc != FSD_OK) return rc;
+        fp.timeout_flag = flags;
+    } else {
+        if (vec) fsd_pair_generic_kernel<DT, true><<<items, 512, 0, s>>>(pp);
+        else     fsd_pair_generic_kernel<DT, false><<<items, 512, 0, s>>>(pp);
+        if (cudaGetLastError() != cudaSuccess) return FSD_ERR_CUDA;
+        fp.timeout_flag = nullptr;
+    }
 
     const int cs = finish_cluster_size(fp.V);
     cudaLaunchConfig_t cfg = {};
@@ -109,12 +180,13 @@ int verify_common(const void* target, const void* draft, const int32_t* tokens, 
     fp.target = target; fp.draft = draft; fp.parent = parent; fp.u_sample = u_sample;
     fp.B = B; fp.G = G; fp.V = V;
     fp.mode = o->mode; fp.sample = o->sample; fp.max_depth = max_depth;
-    fp.item_bits = ws.item_bits; fp.item_status = ws.item_status;
+    fp.item_bits = ws.item_bits; fp.item_status = ws.item_status; fp.timeout_flag = nullptr;
     fp.accept_len = accept_len; fp.path = path; fp.next_token = next_token; fp.row_status = row_status;
 
     const bool vec = (static_cast<size_t>(V) * es) % 16 == 0 && aligned(target, 16) && aligned(draft, 16);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, s) : launch_all<FSD_F32>(pp, fp, vec, s);
+    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, ws.flags, s)
+                                       : launch_all<FSD_F32>(pp, fp, vec, ws.flags, s);
 }
 
 struct HostStaging {

@@ -28,6 +28,7 @@ struct FinishParams {
     int mode, sample, max_depth;
     const int32_t* item_bits;
     const int32_t* item_status;
+    const int* timeout_flag;   // nonzero: a bounded wait of the streaming kernel ran out (may be null)
     int32_t* accept_len;       // [B]
     int32_t* path;             // [B, max_depth] (tree) or null
     int32_t* next_token;       // [B]
@@ -90,6 +91,7 @@ __global__ void __launch_bounds__(kFinishThreads) fsd_finish_kernel(FinishParams
     __syncthreads();
     int st = 0;
     for (int i = tid; i < G; i += blockDim.x) st |= ist[i];
+    if (tid == 0 && P.timeout_flag != nullptr && *P.timeout_flag != 0) st |= FSD_ROW_TIMEOUT;
     st = __reduce_or_sync(0xffffffffu, st);
     if (lane == 0 && st) atomicOr(&sh.bad, st);
     if (P.parent == nullptr) {
