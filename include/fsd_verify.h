@@ -164,13 +164,13 @@ int fsd_verify_chain_host(const void *h_target_logits, const void *h_draft_logit
  * inside another framework's allocator and must not go around it, a serving process whose whole
  * device budget is already handed out.  Such a caller has no buffer to pass as `workspace` and
  * cannot call cudaMalloc to get one.  This variant computes exactly what fsd_verify_chain
- * computes, with the same kernels, but keeps the per-position accept bits and status words in a
- * fixed array that is part of the library's device image, so the caller passes only inputs and
+ * computes, with the same kernels, but keeps the per-position scratch (accept bits, status words
+ * and the 64-byte totals of each position) in a fixed array that is part of the library's device image, so the caller passes only inputs and
  * outputs.  It calls no cudaMalloc, cudaFree or any other allocating routine.
  *
  * Limits and rules
  *   - B * gamma must not exceed FSD_STATIC_MAX_POSITIONS; larger calls are refused with
- *     FSD_ERR_TOO_LARGE and nothing is launched.  The array (FSD_STATIC_SCRATCH_BYTES, 64 KiB)
+ *     FSD_ERR_TOO_LARGE and nothing is launched.  The array (FSD_STATIC_SCRATCH_BYTES, 768 KiB)
  *     is resident on every GPU that loads the library until the process exits.
  *   - The first call on each device looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.
@@ -180,7 +180,7 @@ int fsd_verify_chain_host(const void *h_target_logits, const void *h_draft_logit
  *     them) race on it and give wrong results; order them, or use fsd_verify_chain with
  *     separate workspaces.
  * Arguments, outputs and the other error codes are those of fsd_verify_chain. */
-#define FSD_STATIC_SCRATCH_BYTES 65536
+#define FSD_STATIC_SCRATCH_BYTES 786432
 #define FSD_STATIC_MAX_POSITIONS 8128
 int fsd_verify_chain_static(const void *target_logits, const void *draft_logits,
                             const int32_t *draft_tokens, const float *u_accept, const float *u_sample,

@@ -23,6 +23,7 @@ struct Workspace {
     int32_t* item_bits;
     int32_t* item_status;
     int* flags;                // [0] = a bounded device-side wait ran out
+    PairRecord* records;       // per-pair totals of the streaming kernel
     size_t bytes;
 };
 
@@ -36,6 +37,8 @@ Workspace carve(void* base, int B, int G) {
     p += align_up(items * sizeof(int32_t));
     w.flags = reinterpret_cast<int*>(p);
     p += kAlign;
+    w.records = reinterpret_cast<PairRecord*>(p);
+    p += align_up(items * sizeof(PairRecord));
     w.bytes = static_cast<size_t>(p - static_cast<char*>(base));
     return w;
 }
@@ -96,9 +99,13 @@ int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
             if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
                 return FSD_ERR_CUDA;
+            if (cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+                return FSD_ERR_CUDA;
             cfg.gridDim = dim3(C, 1, 1);
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) return FSD_ERR_CUDA;
+            if (cudaOccupancyMaxActiveClusters(&n, fsd_stream_occupancy_twin, &cfg) != cudaSuccess || n < 1)
+                return FSD_ERR_CUDA;
             max_clusters[dev][lc] = n;
         }
         nclus = max_clusters[dev][lc];
@@ -119,24 +126,27 @@ int stream_cluster_size(int nvec_row, bool vec) {
 }
 
 template <int DT>
-int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, cudaStream_t s) {
+int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, PairRecord* records, cudaStream_t s) {
     const int items = pp.B * pp.G;
     const int nvec_row = pp.V / Logit<DT>::kPerVec;
     const int C = stream_cluster_size(nvec_row, vec);
     if (C > 0) {
         StreamParams sp;
-        sp.pp = pp; sp.nvec_row = nvec_row; sp.n_items = items; sp.timeout_flag = flags;
+        sp.target = pp.target; sp.draft = pp.draft; sp.parent = pp.parent; sp.B = pp.B; sp.G = pp.G;
+        sp.nvec_row = nvec_row; sp.n_items = items; sp.records = records; sp.timeout_flag = flags;
         int rc;
         if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, C, s);
         else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, C, s);
         else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, C, s);
         if (rc != FSD_OK) return rc;
         fp.timeout_flag = flags;
+        fp.records = records;
     } else {
         if (vec) fsd_pair_generic_kernel<DT, true><<<items, 512, 0, s>>>(pp);
         else     fsd_pair_generic_kernel<DT, false><<<items, 512, 0, s>>>(pp);
         if (cudaGetLastError() != cudaSuccess) return FSD_ERR_CUDA;
         fp.timeout_flag = nullptr;
+        fp.records = nullptr;
     }
 
     const int cs = finish_cluster_size(fp.V);
@@ -179,14 +189,17 @@ int verify_common(const void* target, const void* draft, const int32_t* tokens, 
     FinishParams fp;
     fp.target = target; fp.draft = draft; fp.parent = parent; fp.u_sample = u_sample;
     fp.B = B; fp.G = G; fp.V = V;
-    fp.mode = o->mode; fp.sample = o->sample; fp.max_depth = max_depth;
+    fp.tokens = tokens; fp.u_accept = u_accept;
+    fp.div = o->divergence; fp.mode = o->mode; fp.cmp = o->compare; fp.sample = o->sample; fp.max_depth = max_depth;
+    fp.T = o->threshold; fp.records = nullptr; fp.divergence = divergence;
     fp.item_bits = ws.item_bits; fp.item_status = ws.item_status; fp.timeout_flag = nullptr;
     fp.accept_len = accept_len; fp.path = path; fp.next_token = next_token; fp.row_status = row_status;
 
     const bool vec = (static_cast<size_t>(V) * es) % 16 == 0 && aligned(target, 16) && aligned(draft, 16);
+    fp.vec = vec ? 1 : 0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, ws.flags, s)
-                                       : launch_all<FSD_F32>(pp, fp, vec, ws.flags, s);
+    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, ws.flags, ws.records, s)
+                                       : launch_all<FSD_F32>(pp, fp, vec, ws.flags, ws.records, s);
 }
 
 struct HostStaging {

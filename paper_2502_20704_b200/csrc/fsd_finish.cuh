@@ -1,81 +1,165 @@
-// Finish kernel: one thread-block cluster per batch row.  Finds the accepted prefix
-// (chain) or the deepest accepted path (tree) from the per-pair accept bits, then draws
-// the replacement / bonus token from one target row (and, for the SD residual, one
-// draft row) by an inverse CDF in vocabulary order.
+// Finish kernel: one thread-block cluster per batch row.
+//   1. Turns the per-pair totals left by the streaming kernel into divergences and accept
+//      bits (or takes the bits the generic kernel already wrote).
+//   2. Finds the accepted prefix (chain) or the deepest accepted path (tree).
+//   3. Draws the replacement / bonus token from one target row (and, for the SD residual, one
+//      draft row) by an inverse CDF in vocabulary order.
 //
-// The draw must land on the same token as a sequential double-precision sum would, so
-// this kernel evaluates its exponentials and partial sums in double precision: each
-// thread owns a contiguous chunk of the vocabulary, chunk sums are combined by a
-// fixed-order scan (thread -> warp -> CTA -> cluster), the first thread whose inclusive
-// sum exceeds u * total re-walks its chunk.  The rows involved are a 1/(2*gamma+1)
-// share of the logits, and the fp64 pipe is otherwise idle.
+// The draw must land on the same token as a sequential double-precision sum would, so the
+// exponentials and partial sums of step 3 are double precision: each thread owns a contiguous
+// chunk of the vocabulary, chunk sums are combined by a fixed-order scan (thread -> warp ->
+// CTA -> cluster), and the first thread whose inclusive sum exceeds u * total re-walks its
+// chunk.  The double exponential is a 64-entry table times a degree-5 polynomial (about ten
+// fp64 operations); the rows involved are a 1/(2*gamma+1) share of all logits.
 #pragma once
 
 #include "fsd_device.cuh"
+#include "fsd_pair_generic.cuh"
+#include "fsd_pair_stream.cuh"
 
 namespace fsd {
 
 constexpr int kFinishThreads = 512;
-constexpr int kMaxClusterSize = 8;
+constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kMaxTreeNodes = 1024;
 
 struct FinishParams {
     const void* target;        // [B, G+1, V]
     const void* draft;         // [B, G,   V]
     const int32_t* parent;     // tree only
+    const int32_t* tokens;     // [B, G] or null
+    const float* u_accept;     // [B, G] or null
     const float* u_sample;     // [B]
     int B, G, V;
-    int mode, sample, max_depth;
-    const int32_t* item_bits;
-    const int32_t* item_status;
+    int div, mode, cmp, sample, max_depth;
+    int vec;                   // rows are 16-byte aligned and a whole number of vectors
+    float T;
+    const PairRecord* records; // per-pair totals of the streaming kernel, or null (generic kernel ran)
+    int32_t* item_bits;        // [B, G] read when records == null
+    int32_t* item_status;      // [B, G] read when records == null
     const int* timeout_flag;   // nonzero: a bounded wait of the streaming kernel ran out (may be null)
+    float* divergence;         // [B, G] written here when records != null
     int32_t* accept_len;       // [B]
     int32_t* path;             // [B, max_depth] (tree) or null
     int32_t* next_token;       // [B]
     int32_t* row_status;       // [B]
 };
 
+struct FinishExchange {        // what one CTA publishes to its cluster
+    double d[4];
+    int i[2];
+};
 struct FinishShared {
-    double slot_d[2];          // values this CTA publishes to its cluster
-    int slot_i[2];
+    FinishExchange slot;
+    double exp_table[64];      // 2^(j/64)
     double red_d[32 * 2];
     float red_f[32 * 2];
     double warp_tot[32];
     int cand;                  // lowest thread whose inclusive sum exceeds the target
     int last_pos;              // highest index with a positive weight in this CTA
+    int token;
     int row_sel;               // target row the token is drawn from
     int n_acc;
     int bad;
     int16_t tree_depth[kMaxTreeNodes];
     int8_t tree_ok[kMaxTreeNodes];
+    int8_t tree_bit[kMaxTreeNodes];
 };
 
-// Every CTA of the cluster publishes two doubles and two ints and reads everybody's.
-// Two cluster barriers: after the writes, and after the reads (so slots can be reused).
+// 2^y in double precision for y <= 0 (relative error about 2e-16); 0 below the normal range.
+__device__ __forceinline__ double exp2_table(double y, const double* table) {
+    if (!(y > -1000.0)) return y != y ? y : 0.0;
+    const double kMagic = 6755399441055744.0;                      // 1.5 * 2^52: the sum's low word is round(64 y)
+    const double t = fma(y, 64.0, kMagic);
+    const int k = __double2loint(t);
+    const double r = fma(t - kMagic, -1.0 / 64.0, y);              // |r| <= 1/128, exact
+    const double z = r * kLn2D;
+    double p = fma(z, 1.0 / 120.0, 1.0 / 24.0);
+    p = fma(p, z, 1.0 / 6.0);
+    p = fma(p, z, 0.5);
+    p = fma(p, z, 1.0);
+    p = fma(p, z, 1.0);
+    const double m = table[k & 63] * p;                            // in [1, 2.0001)
+    const int hi = __double2hiint(m) + ((k >> 6) << 20);           // scale by 2^(k >> 6): stays normal for y > -1000
+    return __hiloint2double(hi, __double2loint(m));
+}
+
+// Every CTA of the cluster publishes a FinishExchange and reads everybody's.
+// Two cluster barriers: after the writes, and after the reads (so the slot can be reused).
 __device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, FinishShared& sh, int cs,
-                                                 double d0, double d1, int i0, int i1,
-                                                 double (&od0)[kMaxClusterSize], double (&od1)[kMaxClusterSize],
-                                                 int (&oi0)[kMaxClusterSize], int (&oi1)[kMaxClusterSize]) {
-    if (threadIdx.x == 0) {
-        sh.slot_d[0] = d0; sh.slot_d[1] = d1;
-        sh.slot_i[0] = i0; sh.slot_i[1] = i1;
-    }
+                                                 const FinishExchange& mine, FinishExchange (&all)[kMaxClusterSize]) {
+    if (threadIdx.x == 0) sh.slot = mine;
     cluster.sync();
 #pragma unroll
     for (int r = 0; r < kMaxClusterSize; ++r) {
-        if (r < cs) {
-            const FinishShared* rs = cluster.map_shared_rank(&sh, r);
-            od0[r] = rs->slot_d[0]; od1[r] = rs->slot_d[1];
-            oi0[r] = rs->slot_i[0]; oi1[r] = rs->slot_i[1];
-        } else {
-            od0[r] = 0.0; od1[r] = 0.0; oi0[r] = 0; oi1[r] = 0;
-        }
+        if (r < cs) all[r] = cluster.map_shared_rank(&sh, r)->slot;
     }
     cluster.sync();
 }
 
+// Divergence, accept bit and status of one pair from the streaming kernel's totals.
+__device__ inline void judge_record(const FinishParams& P, int item, const void* a_row, const void* b_row, int dt,
+                                    float& D_out, int& bit_out, int& st_out) {
+    const PairRecord r = P.records[item];
+    if (r.state & kRecordBadTree) {
+        D_out = __int_as_float(0x7fc00000); bit_out = 0; st_out = FSD_ROW_BADTREE;
+        return;
+    }
+    const bool finite = isfinite(r.ka) && isfinite(r.kb) && r.Za > 0.0 && r.Zb > 0.0 && isfinite(r.Za) && isfinite(r.Zb);
+    float D = __int_as_float(0x7fc00000);
+    if (finite) D = r.differ ? static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X)) : 0.0f;
+    const bool div_ok = finite && passes(D, P.T, P.cmp);
+    int bit = div_ok;
+    if (P.mode != FSD_MODE_FSD) {
+        bool ratio_ok = false;
+        if (finite) {
+            const int x = P.tokens[item];
+            if (x >= 0 && x < P.V) {
+                const float ax = dt == FSD_BF16 ? load_logit<FSD_BF16>(a_row, x) : load_logit<FSD_F32>(a_row, x);
+                const float bx = dt == FSD_BF16 ? load_logit<FSD_BF16>(b_row, x) : load_logit<FSD_F32>(b_row, x);
+                double pacc;                                                    // Eq. 1
+                if (bx == -INFINITY) {
+                    pacc = (ax != -INFINITY) ? 1.0 : 0.0;
+                } else {
+                    // ln P(x) = (x*log2e - k) ln2 - ln Z with the same float log2e the sums were built with
+                    const double la = (static_cast<double>(ax) * static_cast<double>(kLog2e) - r.ka) * kLn2D - log(r.Za);
+                    const double lb = (static_cast<double>(bx) * static_cast<double>(kLog2e) - r.kb) * kLn2D - log(r.Zb);
+                    pacc = exp(la - lb);
+                    pacc = pacc < 1.0 ? pacc : 1.0;
+                }
+                ratio_ok = static_cast<double>(P.u_accept[item]) < pacc;        // Eq. 2
+            }
+        }
+        bit = P.mode == FSD_MODE_SD ? ratio_ok : (div_ok || ratio_ok);          // Eq. 6
+    }
+    D_out = D; bit_out = bit; st_out = finite ? 0 : FSD_ROW_NONFINITE;
+}
+
+// Calls f(k, a_k, b_k) for k in [k0, k1) in order; 16-byte loads when `vec` (then k0 is a
+// multiple of the vector width and V a multiple of it).  b_k is 0 unless `with_b`.
+template <int DT, typename F>
+__device__ __forceinline__ void for_chunk(const void* a_row, const void* b_row, int k0, int k1, bool vec, bool with_b, F f) {
+    constexpr int EPV = Logit<DT>::kPerVec;
+    if (vec) {
+        for (int k = k0; k < k1; k += EPV) {
+            float xa[EPV], xb[EPV];
+            unpack_vec<DT>(ldg_vec(a_row, k / EPV), xa);
+            if (with_b) {
+                unpack_vec<DT>(ldg_vec(b_row, k / EPV), xb);
+            } else {
+#pragma unroll
+                for (int j = 0; j < EPV; ++j) xb[j] = 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) f(k + j, xa[j], xb[j]);
+        }
+    } else {
+        for (int k = k0; k < k1; ++k) f(k, load_logit<DT>(a_row, k), with_b ? load_logit<DT>(b_row, k) : 0.f);
+    }
+}
+
 template <int DT>
-__global__ void __launch_bounds__(kFinishThreads) fsd_finish_kernel(FinishParams P) {
+__global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishParams P) {
     __shared__ FinishShared sh;
     cg::cluster_group cluster = cg::this_cluster();
     const int cs = static_cast<int>(cluster.num_blocks());
@@ -83,35 +167,58 @@ __global__ void __launch_bounds__(kFinishThreads) fsd_finish_kernel(FinishParams
     const int b = blockIdx.x / cs;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = P.G, V = P.V;
-    const int32_t* bits = P.item_bits + static_cast<size_t>(b) * G;
-    const int32_t* ist = P.item_status + static_cast<size_t>(b) * G;
+    const size_t rb = static_cast<size_t>(V) * Logit<DT>::kBytes;
+    const char* t_base = static_cast<const char*>(P.target) + static_cast<size_t>(b) * (G + 1) * rb;
+    const char* d_base = static_cast<const char*>(P.draft) + static_cast<size_t>(b) * G * rb;
+    const bool tree = P.parent != nullptr;
 
-    // ---- accepted prefix / accepted path (every CTA computes it; rank 0 writes it) ----
-    if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; }
+    if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; sh.token = -1; }
+    if (tid < 64) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / 64.0));
     __syncthreads();
-    int st = 0;
-    for (int i = tid; i < G; i += blockDim.x) st |= ist[i];
+
+    // ---- 1. divergences, accept bits, status of this row's pairs ----
+    int st = 0, first = G;
+    for (int i = tid; i < G; i += blockDim.x) {
+        const int item = b * G + i;
+        int bit, s;
+        if (P.records != nullptr) {
+            int trow = i;
+            if (tree) {
+                const int par = P.parent[item];
+                trow = (par >= -1 && par < i) ? par + 1 : 0;
+            }
+            float D;
+            judge_record(P, item, t_base + static_cast<size_t>(trow) * rb, d_base + static_cast<size_t>(i) * rb, DT, D, bit, s);
+            if (rank == 0) P.divergence[item] = D;
+        } else {
+            bit = P.item_bits[item];
+            s = P.item_status[item];
+        }
+        st |= s;
+        if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
+        else if (!bit && i < first) first = i;
+    }
     if (tid == 0 && P.timeout_flag != nullptr && *P.timeout_flag != 0) st |= FSD_ROW_TIMEOUT;
     st = __reduce_or_sync(0xffffffffu, st);
-    if (lane == 0 && st) atomicOr(&sh.bad, st);
-    if (P.parent == nullptr) {
-        int first = G;
-        for (int i = tid; i < G; i += blockDim.x)
-            if (!bits[i]) { first = i; break; }
-        first = __reduce_min_sync(0xffffffffu, first);
-        if (lane == 0) atomicMin(&sh.n_acc, first);
-        __syncthreads();
-        if (tid == 0) sh.row_sel = sh.n_acc;
-    } else {
-        __syncthreads();
-        if (tid == 0) {
+    first = __reduce_min_sync(0xffffffffu, first);
+    if (lane == 0) {
+        if (st) atomicOr(&sh.bad, st);
+        if (!tree) atomicMin(&sh.n_acc, first);
+    }
+    __syncthreads();
+
+    // ---- 2. accepted prefix (chain) or deepest accepted path (tree) ----
+    if (tid == 0) {
+        if (!tree) {
+            sh.row_sel = sh.n_acc;
+        } else {
             const int32_t* par = P.parent + static_cast<size_t>(b) * G;
             int best = -1, best_depth = 0;
             if (!(sh.bad & FSD_ROW_BADTREE)) {
                 for (int j = 0; j < G; ++j) {
                     const int p = par[j];
                     const int d = p < 0 ? 1 : sh.tree_depth[p] + 1;
-                    const bool ok = bits[j] && (p < 0 || sh.tree_ok[p]);
+                    const bool ok = sh.tree_bit[j] && (p < 0 || sh.tree_ok[p]);
                     sh.tree_depth[j] = static_cast<int16_t>(d);
                     sh.tree_ok[j] = ok;
                     if (ok && d <= P.max_depth && d > best_depth) { best = j; best_depth = d; }
@@ -130,84 +237,123 @@ __global__ void __launch_bounds__(kFinishThreads) fsd_finish_kernel(FinishParams
     const int n = sh.n_acc, row_sel = sh.row_sel;
     int status = sh.bad;
     if (status & FSD_ROW_BADTREE) {                      // uniform over the cluster
-        if (rank == 0 && tid == 0) {
-            P.accept_len[b] = 0;
-            P.next_token[b] = -1;
-            P.row_status[b] = status;
-        }
+        if (rank == 0 && tid == 0) { P.accept_len[b] = 0; P.next_token[b] = -1; P.row_status[b] = status; }
         return;
     }
-    const bool residual0 = (P.mode != FSD_MODE_FSD) && P.parent == nullptr && n < G;
 
-    const size_t rb = static_cast<size_t>(V) * Logit<DT>::kBytes;
-    const char* a_row = static_cast<const char*>(P.target) + (static_cast<size_t>(b) * (G + 1) + row_sel) * rb;
-    const char* b_row = static_cast<const char*>(P.draft) + (static_cast<size_t>(b) * G + (residual0 ? n : 0)) * rb;
+    // ---- 3. token draw ----
+    constexpr int EPV = Logit<DT>::kPerVec;
+    const bool vec = P.vec != 0;
+    const bool residual0 = (P.mode != FSD_MODE_FSD) && !tree && n < G;
+    const bool greedy = P.sample == FSD_SAMPLE_GREEDY;
+    const char* a_row = t_base + static_cast<size_t>(row_sel) * rb;
+    const char* b_row = d_base + static_cast<size_t>(residual0 ? n : 0) * rb;
+    const double* tab = sh.exp_table;
 
     // contiguous chunk of the vocabulary owned by this thread
     const int tt = cs * blockDim.x;
-    const int L = (V + tt - 1) / tt;
-    const int g = rank * blockDim.x + tid;
-    const long long k0l = static_cast<long long>(g) * L;
+    const int L = vec ? ((V / EPV + tt - 1) / tt) * EPV : (V + tt - 1) / tt;
+    const long long k0l = static_cast<long long>(rank * blockDim.x + tid) * L;
     const int k0 = k0l < V ? static_cast<int>(k0l) : V;
     const int k1 = (k0l + L) < V ? static_cast<int>(k0l + L) : V;
+    FinishExchange mine, all[kMaxClusterSize];
 
-    double xd0[kMaxClusterSize], xd1[kMaxClusterSize];
-    int xi0[kMaxClusterSize], xi1[kMaxClusterSize];
-
-    // ---- maxima (exact) and, for the greedy FSD choice, the argmax of the logits ----
+    // ---- CTA-local maxima (exact); for the greedy FSD choice also the argmax of the logits ----
     float mx[2] = {-INFINITY, -INFINITY};
     int amax = 0x7fffffff;
-    for (int k = k0; k < k1; ++k) {
-        const float a = load_logit<DT>(a_row, k);
-        if (a > mx[0]) { mx[0] = a; amax = k; }
-        if (residual0) mx[1] = fmaxf(mx[1], load_logit<DT>(b_row, k));
-    }
-    const float my_max = mx[0];
+    float amax_v = -INFINITY;
+    for_chunk<DT>(a_row, b_row, k0, k1, vec, residual0, [&](int k, float xa, float xb) {
+        if (xa > amax_v) { amax_v = xa; amax = k; }
+        mx[1] = fmaxf(mx[1], xb);
+    });
+    mx[0] = amax_v;
     block_max<2>(mx, sh.red_f);
-    cluster_exchange(cluster, sh, cs, mx[0], mx[1], 0, 0, xd0, xd1, xi0, xi1);
-    double Ma = -INFINITY, Mb = -INFINITY;
-    for (int r = 0; r < cs; ++r) { Ma = fmax(Ma, xd0[r]); Mb = fmax(Mb, xd1[r]); }
+    const double Ra = mx[0], Rb = mx[1];                 // this CTA's references
 
-    // ---- normalisers in double ----
-    double z[2] = {0.0, 0.0};
-    for (int k = k0; k < k1; ++k) {
-        z[0] += exp(static_cast<double>(load_logit<DT>(a_row, k)) - Ma);
-        if (residual0) z[1] += exp(static_cast<double>(load_logit<DT>(b_row, k)) - Mb);
-    }
-    block_sum<2>(z, sh.red_d);
-    cluster_exchange(cluster, sh, cs, z[0], z[1], 0, 0, xd0, xd1, xi0, xi1);
-    double Za = 0.0, Zb = 0.0;
-    for (int r = 0; r < cs; ++r) { Za += xd0[r]; Zb += xd1[r]; }
-    const bool a_ok = isfinite(Ma) && isfinite(Za) && Za > 0.0;
-    bool residual = residual0 && isfinite(Mb) && isfinite(Zb) && Zb > 0.0;
-    if (!a_ok) {                                          // uniform over the cluster
+    if (greedy && !residual0) {
+        // argmax of P_T == argmax of the logits, ties to the lowest index
+        float best = amax_v;
+        int idx = amax;
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, m);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, m);
+            if (ob > best || (ob == best && oi < idx)) { best = ob; idx = oi; }
+        }
+        if (lane == 0) { sh.red_d[warp * 2] = best; sh.red_d[warp * 2 + 1] = idx; }
+        __syncthreads();
+        best = static_cast<float>(sh.red_d[0]); idx = static_cast<int>(sh.red_d[1]);
+        for (int w = 1; w < kFinishWarps; ++w) {
+            const float ob = static_cast<float>(sh.red_d[w * 2]);
+            const int oi = static_cast<int>(sh.red_d[w * 2 + 1]);
+            if (ob > best || (ob == best && oi < idx)) { best = ob; idx = oi; }
+        }
+        // a NaN or +inf logit, or no finite logit, makes the row invalid: detect through the sum of the logits' signs
+        float bad_v = 0.f;
+        for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int, float xa, float) { if (xa != xa || xa == INFINITY) bad_v = 1.f; });
+        float bv[1] = {bad_v};
+        block_max<1>(bv, sh.red_f);
+        mine.d[0] = best; mine.d[1] = bv[0]; mine.d[2] = 0; mine.d[3] = 0; mine.i[0] = idx; mine.i[1] = 0;
+        cluster_exchange(cluster, sh, cs, mine, all);
+        double gb = all[0].d[0], gbad = all[0].d[1];
+        int gi = all[0].i[0];
+        for (int r = 1; r < cs; ++r) {
+            if (all[r].d[0] > gb || (all[r].d[0] == gb && all[r].i[0] < gi)) { gb = all[r].d[0]; gi = all[r].i[0]; }
+            gbad = fmax(gbad, all[r].d[1]);
+        }
+        const bool ok = gbad == 0.0 && gb > -INFINITY;
         if (rank == 0 && tid == 0) {
             P.accept_len[b] = n;
-            P.next_token[b] = -1;
-            P.row_status[b] = status | FSD_ROW_NONFINITE;
+            P.next_token[b] = ok ? gi : -1;
+            P.row_status[b] = status | (ok ? 0 : FSD_ROW_NONFINITE);
         }
         return;
     }
-    const double iZa = 1.0 / Za, iZb = residual ? 1.0 / Zb : 0.0;
-    auto weight = [&](int k, bool res) -> double {
-        const double ea = exp(static_cast<double>(load_logit<DT>(a_row, k)) - Ma);
-        if (!res) return ea;
-        const double r = ea * iZa - exp(static_cast<double>(load_logit<DT>(b_row, k)) - Mb) * iZb;
-        return r > 0.0 ? r : 0.0;
-    };
 
-    int token = -1;
+    // ---- residual only: global normalisers of both rows (double) ----
+    double Ma = Ra, Mb = Rb, iZa = 0.0, iZb = 0.0;
+    bool residual = residual0;
+    if (residual0) {
+        double z[2] = {0.0, 0.0};
+        for_chunk<DT>(a_row, b_row, k0, k1, vec, true, [&](int, float xa, float xb) {
+            if (Ra > -INFINITY) z[0] += exp2_table((static_cast<double>(xa) - Ra) * kLog2eD, tab);
+            if (Rb > -INFINITY) z[1] += exp2_table((static_cast<double>(xb) - Rb) * kLog2eD, tab);
+        });
+        block_sum<2>(z, sh.red_d);
+        mine.d[0] = Ra; mine.d[1] = Rb; mine.d[2] = z[0]; mine.d[3] = z[1]; mine.i[0] = 0; mine.i[1] = 0;
+        cluster_exchange(cluster, sh, cs, mine, all);
+        Ma = -INFINITY; Mb = -INFINITY;
+        for (int r = 0; r < cs; ++r) { Ma = fmax(Ma, all[r].d[0]); Mb = fmax(Mb, all[r].d[1]); }
+        double Za = 0.0, Zb = 0.0;
+        for (int r = 0; r < cs; ++r) {
+            if (all[r].d[0] > -INFINITY) Za += all[r].d[2] * exp2_table((all[r].d[0] - Ma) * kLog2eD, tab);
+            if (all[r].d[1] > -INFINITY) Zb += all[r].d[3] * exp2_table((all[r].d[1] - Mb) * kLog2eD, tab);
+        }
+        const bool a_ok = isfinite(Ma) && isfinite(Za) && Za > 0.0, b_ok = isfinite(Mb) && isfinite(Zb) && Zb > 0.0;
+        if (!a_ok) {                                      // uniform over the cluster
+            if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.next_token[b] = -1; P.row_status[b] = status | FSD_ROW_NONFINITE; }
+            return;
+        }
+        if (!b_ok) { residual = false; status |= FSD_ROW_NONFINITE; }
+        else { iZa = 1.0 / Za; iZb = 1.0 / Zb; }
+    }
+
     for (int attempt = 0; attempt < 2; ++attempt) {
-        // chunk sum, last positive index and (greedy) the largest weight of the chunk
+        // weight of one vocabulary entry: P_T relative to this CTA's maximum, or the SD residual
+        auto weight = [&](float xa, float xb) -> double {
+            if (!residual) return Ra > -INFINITY ? exp2_table((static_cast<double>(xa) - Ra) * kLog2eD, tab) : 0.0;
+            const double r = exp2_table((static_cast<double>(xa) - Ma) * kLog2eD, tab) * iZa -
+                             exp2_table((static_cast<double>(xb) - Mb) * kLog2eD, tab) * iZb;
+            return r > 0.0 ? r : 0.0;
+        };
         double csum = 0.0, wbest = 0.0;
         int lastp = -1, kbest = 0x7fffffff;
-        const bool need_w = residual || P.sample != FSD_SAMPLE_GREEDY;
-        for (int k = k0; need_w && k < k1; ++k) {
-            const double w = weight(k, residual);
+        for_chunk<DT>(a_row, b_row, k0, k1, vec, residual, [&](int k, float xa, float xb) {
+            const double w = weight(xa, xb);
             csum += w;
             if (w > 0.0) lastp = k;
             if (w > wbest) { wbest = w; kbest = k; }
-        }
+        });
         // inclusive / exclusive scan of the chunk sums over the CTA, fixed order
         double incl = csum;
 #pragma unroll
@@ -218,103 +364,99 @@ __global__ void __launch_bounds__(kFinishThreads) fsd_finish_kernel(FinishParams
         double excl = __shfl_up_sync(0xffffffffu, incl, 1);
         if (lane == 0) excl = 0.0;
         if (lane == 31) sh.warp_tot[warp] = incl;
+        if (greedy) {                                     // residual arg-max of the warp, ties to the lowest index
+#pragma unroll
+            for (int m = 16; m > 0; m >>= 1) {
+                const double ob = shfl_xor_d(wbest, m);
+                const int oi = __shfl_xor_sync(0xffffffffu, kbest, m);
+                if (ob > wbest || (ob == wbest && oi < kbest)) { wbest = ob; kbest = oi; }
+            }
+            if (lane == 0) { sh.red_d[warp * 2] = wbest; sh.red_d[warp * 2 + 1] = kbest; }
+        }
+        const int lp = __reduce_max_sync(0xffffffffu, lastp);
+        if (lane == 0 && lp >= 0) atomicMax(&sh.last_pos, lp);
         __syncthreads();
         double wpre = 0.0, cta_tot = 0.0;
-        const int nwarps = blockDim.x >> 5;
-        for (int w = 0; w < nwarps; ++w) {
+        for (int w = 0; w < kFinishWarps; ++w) {
             if (w == warp) wpre = cta_tot;
             cta_tot += sh.warp_tot[w];
         }
         incl += wpre;
         excl += wpre;
-
-        if (P.sample == FSD_SAMPLE_GREEDY) {
-            // FSD: argmax of p == argmax of the logits; residual: argmax of max(0, p - q)
-            double best = residual ? wbest : static_cast<double>(my_max);
-            int idx = residual ? kbest : amax;
-            // block arg-max with ties to the lowest index
-#pragma unroll
-            for (int m = 16; m > 0; m >>= 1) {
-                const double ob = shfl_xor_d(best, m);
-                const int oi = __shfl_xor_sync(0xffffffffu, idx, m);
-                if (ob > best || (ob == best && oi < idx)) { best = ob; idx = oi; }
-            }
-            __syncthreads();
-            if (lane == 0) { sh.red_d[warp * 2] = best; sh.red_d[warp * 2 + 1] = static_cast<double>(idx); }
-            __syncthreads();
-            best = sh.red_d[0];
-            idx = static_cast<int>(sh.red_d[1]);
-            for (int w = 1; w < nwarps; ++w) {
+        if (greedy) {
+            wbest = sh.red_d[0]; kbest = static_cast<int>(sh.red_d[1]);
+            for (int w = 1; w < kFinishWarps; ++w) {
                 const double ob = sh.red_d[w * 2];
                 const int oi = static_cast<int>(sh.red_d[w * 2 + 1]);
-                if (ob > best || (ob == best && oi < idx)) { best = ob; idx = oi; }
+                if (ob > wbest || (ob == wbest && oi < kbest)) { wbest = ob; kbest = oi; }
             }
-            cluster_exchange(cluster, sh, cs, best, cta_tot, idx, 0, xd0, xd1, xi0, xi1);
-            double tot = 0.0;
-            for (int r = 0; r < cs; ++r) tot += xd1[r];
-            if (residual && !(tot > 0.0)) { residual = false; continue; }   // no residual mass: use P_T
-            best = xd0[0]; idx = xi0[0];
-            for (int r = 1; r < cs; ++r)
-                if (xd0[r] > best || (xd0[r] == best && xi0[r] < idx)) { best = xd0[r]; idx = xi0[r]; }
-            token = idx;
-            break;
         }
+        mine.d[0] = cta_tot; mine.d[1] = Ra; mine.d[2] = wbest; mine.d[3] = 0; mine.i[0] = sh.last_pos; mine.i[1] = kbest;
+        cluster_exchange(cluster, sh, cs, mine, all);
 
-        // highest positive index of this CTA (fallback when rounding leaves no crossing)
-        int lp = __reduce_max_sync(0xffffffffu, lastp);
-        if (lane == 0 && lp >= 0) atomicMax(&sh.last_pos, lp);
-        __syncthreads();
-        cluster_exchange(cluster, sh, cs, cta_tot, 0.0, sh.last_pos, 0, xd0, xd1, xi0, xi1);
-        double W = 0.0;
-        for (int r = 0; r < cs; ++r) W += xd0[r];
-        if (residual && !(W > 0.0)) {                     // no residual mass: use P_T (uniform decision)
+        // cluster totals on a common reference
+        double M = -INFINITY;
+        for (int r = 0; r < cs; ++r) M = fmax(M, all[r].d[1]);
+        double sc[kMaxClusterSize], W = 0.0;
+        for (int r = 0; r < cs; ++r) {
+            sc[r] = residual ? 1.0 : (all[r].d[1] > -INFINITY ? exp2_table((all[r].d[1] - M) * kLog2eD, tab) : 0.0);
+            W += all[r].d[0] * sc[r];
+        }
+        if (residual && !(W > 0.0)) {                     // no residual mass: draw from P_T (uniform decision)
             residual = false;
+            __syncthreads();
             if (tid == 0) sh.last_pos = -1;
             __syncthreads();
             continue;
         }
+        if (!residual && !(isfinite(M) && isfinite(W) && W > 0.0)) {     // uniform over the cluster
+            if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.next_token[b] = -1; P.row_status[b] = status | FSD_ROW_NONFINITE; }
+            return;
+        }
+        if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.row_status[b] = status; }
+
+        if (greedy) {                                     // residual arg-max over the cluster
+            double gb = all[0].d[2];
+            int gi = all[0].i[1];
+            for (int r = 1; r < cs; ++r)
+                if (all[r].d[2] > gb || (all[r].d[2] == gb && all[r].i[1] < gi)) { gb = all[r].d[2]; gi = all[r].i[1]; }
+            if (rank == 0 && tid == 0) P.next_token[b] = gi;
+            return;
+        }
+
         const double t = static_cast<double>(P.u_sample[b]) * W;
-        // the CTA whose inclusive total first exceeds t
         double cpre = 0.0, run = 0.0;
         int owner = -1, last_any = -1;
         for (int r = 0; r < cs; ++r) {
-            if (r == rank) cpre = run;
-            run += xd0[r];
-            if (owner < 0 && run > t) owner = r;
-            if (xi0[r] > last_any) last_any = xi0[r];
-        }
-        int result = -1;
-        if (owner < 0) {
-            result = last_any;                            // t >= W after rounding: last token with weight
-        } else if (owner == rank) {
-            if (csum > 0.0 && cpre + incl > t) atomicMin(&sh.cand, tid);
-            __syncthreads();
-            const int c = sh.cand;
-            if (c == 0x7fffffff) {
-                if (tid == 0) sh.slot_i[1] = sh.last_pos; // crossing lost to rounding inside this CTA
-            } else if (tid == c) {
-                double running = cpre + excl;
-                int tok = lastp;
-                for (int k = k0; k < k1; ++k) {
-                    running += weight(k, residual);
-                    if (running > t) { tok = k; break; }
-                }
-                sh.slot_i[1] = tok;
+            if (owner < 0) {
+                cpre = run;
+                run += all[r].d[0] * sc[r];
+                if (run > t) owner = r;
             }
-            __syncthreads();
-            result = sh.slot_i[1];
+            if (all[r].i[0] > last_any) last_any = all[r].i[0];
         }
-        // publish the owner's result to the cluster
-        cluster_exchange(cluster, sh, cs, 0.0, 0.0, result, 0, xd0, xd1, xi0, xi1);
-        token = owner < 0 ? result : xi0[owner];
-        break;
-    }
-
-    if (rank == 0 && tid == 0) {
-        P.accept_len[b] = n;
-        P.next_token[b] = token;
-        P.row_status[b] = status | ((residual0 && !(isfinite(Mb) && isfinite(Zb) && Zb > 0.0)) ? FSD_ROW_NONFINITE : 0);
+        if (owner < 0) {                                  // t >= W after rounding: the last token that has weight
+            if (rank == 0 && tid == 0) P.next_token[b] = last_any;
+            return;
+        }
+        if (owner != rank) return;
+        const double t_local = (t - cpre) / sc[owner];    // the target on this CTA's own scale
+        if (csum > 0.0 && incl > t_local) atomicMin(&sh.cand, tid);
+        __syncthreads();
+        const int c = sh.cand;
+        if (c == 0x7fffffff) {                            // crossing lost to rounding inside this CTA
+            if (tid == 0) P.next_token[b] = sh.last_pos;
+        } else if (tid == c) {
+            double running = excl;
+            int tok = lastp;
+            bool found = false;
+            for_chunk<DT>(a_row, b_row, k0, k1, vec, residual, [&](int k, float xa, float xb) {
+                running += weight(xa, xb);
+                if (!found && running > t_local) { tok = k; found = true; }
+            });
+            P.next_token[b] = tok;
+        }
+        return;
     }
 }
-
 }  // namespace fsd

@@ -7,21 +7,23 @@
 //      copies (cp.async.bulk + mbarrier; the next pair's slices stream in meanwhile),
 //   2. sweeps the slice once from shared memory for each thread's exact maximum and a
 //      bitwise "rows differ" flag,
-//   3. sweeps it again computing e = 2^(log2e * (logit - thread max)) with one MUFU ex2 per
-//      logit, the sums Z = sum e and S = sum e*y (and the KL sum), and parks the e values in
-//      tensor memory (64 per thread) and registers (16 per thread),
-//   4. combines (max, Z, S) over threads, warps, CTA and -- through distributed shared memory
-//      and one cluster barrier -- the cluster,
-//   5. sweeps the parked e values: p = e_a/Z_a, q = e_b/Z_b, JS needs sum (p+q) log2(p+q) (one
+//   3. sweeps it again computing e = 2^(logit * log2e - k) with one MUFU ex2 per logit, where k
+//      is the thread's maximum rounded up to an integer in the log2 domain (so every later
+//      change of reference is an exact power of two), the sums Z = sum e and S = sum e*y (and
+//      the KL sum), and parks the e values in tensor memory (64 per thread) and registers (16),
+//   4. combines (k, Z, S) over threads and warps, then -- one CTA barrier and one cluster
+//      barrier later -- over the CTA and, through distributed shared memory, the cluster,
+//   5. sweeps the parked e values: p = e_a/Z_a, q = e_b/Z_b; JS needs sum (p+q) log2(p+q) (one
 //      MUFU lg2 per pair), TV needs sum |p - q|; KL needs no second sweep.
-// The logits themselves are never touched again after step 3, so HBM traffic is the
-// algorithmic minimum; the special-function pipe (1 ex2 per logit + 1 lg2 per pair) is the
-// co-bottleneck, which is why e values are kept rather than recomputed.
-// Two CTAs share an SM so that one CTA's reduction / barrier bubbles are filled by the other.
+// The cluster's rank-0 CTA writes the pair's totals to a 64-byte record; the finish kernel
+// turns records into divergences and accept bits, so no double-precision transcendental runs
+// here.  The logits are never touched again after step 3: HBM traffic is the algorithmic
+// minimum.  The special-function pipe (1 ex2 per logit + 1 lg2 per pair) is the co-bottleneck,
+// which is why e values are kept rather than recomputed.  Two CTAs share an SM so that one
+// CTA's barrier bubbles are filled by the other.
 #pragma once
 
 #include "fsd_device.cuh"
-#include "fsd_pair_generic.cuh"
 
 namespace fsd {
 
@@ -34,13 +36,30 @@ constexpr int kMaxStagesPerPair = kRing - 1;               // a pair's slice mus
 constexpr int kTmemCols = 256;                             // per CTA: 16 warps -> 4 per lane quarter x 64 columns
 constexpr int kTmemPerThread = 64;
 constexpr int kMaxVecPerCta = kMaxStagesPerPair * kStreamThreads;
+constexpr int kMaxClusterSize = 8;
 constexpr uint32_t kSpinLimit = 1u << 24;                  // polls before a wait gives up
 
+// Totals of one pair, written by the streaming kernel and read by the finish kernel.
+//   Z = sum 2^y, S = sum 2^y * y, K = sum 2^ya (ya - yb), with y = logit*log2e - k and k the
+//   integer reference of the row; X = second-sweep sum (JS: sum s log2 s, TV: sum |p - q|).
+struct PairRecord {
+    double Za, Zb, Sa, Sb, K, X;
+    float ka, kb;              // integer-valued references (log2 domain); -inf: no finite logit; NaN: row holds a NaN
+    uint32_t differ;           // 0: the two rows are bitwise identical
+    uint32_t state;            // kRecordStats | kRecordBadTree
+};
+static_assert(sizeof(PairRecord) == 64, "PairRecord is one 64-byte line");
+constexpr uint32_t kRecordStats = 1, kRecordBadTree = 2;
+
 struct StreamParams {
-    PairParams pp;
+    const void* target;        // [B, G+1, V]
+    const void* draft;         // [B, G,   V]
+    const int32_t* parent;     // [B, G] (tree) or null (chain)
+    int B, G;
     int nvec_row;              // 16-byte vectors per logit row
     int n_items;               // B * G
-    int* timeout_flag;         // set to 1 if a bounded wait ran out (host reports FSD_ROW_TIMEOUT)
+    PairRecord* records;       // [B * G]
+    int* timeout_flag;         // set to 1 if a bounded wait ran out
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -109,9 +128,14 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // NaN-propagating maxima: a NaN logit must reach the row maximum so that the row is flagged
-__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+__device__ __forceinline__ uint32_t bf16x2_max_nan(uint32_t a, uint32_t b) {
     uint32_t d;
     asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
 __device__ __forceinline__ float fmax_nan(float a, float b) {
@@ -124,63 +148,36 @@ __device__ __forceinline__ float warp_max_nan(float v) {
     for (int m = 16; m > 0; m >>= 1) v = fmax_nan(v, __shfl_xor_sync(0xffffffffu, v, m));
     return v;
 }
+// 2^d for an integer-valued d <= 0 (exact); 0 below the normal range and for d = -inf; NaN for NaN
+__device__ __forceinline__ float pow2_int(float d) {
+    if (d != d) return d;
+    return d < -126.f ? 0.f : __int_as_float((static_cast<int>(d) + 127) << 23);
+}
 
 // ---- shared-memory layout ---------------------------------------------------------------
 struct WarpStats {             // one per warp, written by lane 0 after the exponential sweep
-    float ra, rb;              // warp reference (maximum logit) of each row
-    float za, zb, sa, sb, kk;  // sums relative to the warp reference
+    float ka, kb;              // warp references
+    float za, zb, sa, sb, kk;  // sums relative to the warp references
+    float x;                   // second-sweep sum of the PREVIOUS pair
     uint32_t diff;
 };
 struct CtaStats {              // one per CTA and parity, read by the whole cluster
-    float ra, rb;
-    double za, zb, sa, sb, kk;
-    double x_prev;             // second-sweep sum of the PREVIOUS pair
+    float ka, kb;
+    float za, zb, sa, sb, kk;
+    float x;
     uint32_t diff;
-};
-struct Pending {               // what rank 0 needs to finish a pair once its second-sweep sum arrives
-    int item;                  // -1 = nothing pending
-    int finite, differ;
-    float Ma, Mb;              // row maxima
-    double Za, Zb, Sa, Sb, K;  // totals relative to the maxima
 };
 struct StreamShared {
     uint64_t full[kRing];
     uint64_t empty[kRing];
     uint32_t tmem_base;
-    float bc_Ma, bc_Mb, bc_iZa, bc_iZb;    // broadcast of the pair's maxima and reciprocal normalisers
+    // producer cursor (thread 0 only; kept here to spare registers)
+    int p_item, p_stage;
+    uint32_t p_g;
     WarpStats ws[kStreamWarps];
-    float wx[kStreamWarps];                // per-warp second-sweep sums
     CtaStats xch[2];
-    Pending pend;                          // written by warp 0, consumed by the last warp (rank 0 only)
 };
 constexpr size_t kStreamSmemBytes = kRing * kStageBytes + sizeof(StreamShared) + 128;
-
-// ---- final scalar work of one pair (rank 0, one thread) --------------------------------
-__device__ inline void finish_pair(const StreamParams& P, const Pending& pd, double X, int dt) {
-    const PairParams& pp = P.pp;
-    const int item = pd.item;
-    float D = __int_as_float(0x7fc00000);
-    if (pd.finite) {
-        D = pd.differ ? static_cast<float>(combine_divergence(pp.div, pd.Za, pd.Zb, pd.Sa, pd.Sb, pd.K, X)) : 0.0f;
-    }
-    pp.divergence[item] = D;
-    const int b = item / pp.G, i = item - b * pp.G;
-    int trow = i;
-    if (pp.parent != nullptr) trow = pp.parent[item] + 1;
-    const size_t rb = static_cast<size_t>(pp.V) * (dt == FSD_BF16 ? 2 : 4);
-    const char* a_row = static_cast<const char*>(pp.target) + (static_cast<size_t>(b) * (pp.G + 1) + trow) * rb;
-    const char* b_row = static_cast<const char*>(pp.draft) + (static_cast<size_t>(b) * pp.G + i) * rb;
-    // the sums are relative to the exact maxima, so the offsets used are exactly -M*log2e in double
-    const float ca = -pd.Ma * kLog2e, cb = -pd.Mb * kLog2e;
-    double Za = pd.Za, Zb = pd.Zb;
-    if (pd.finite) {
-        // log_prob() expects Z accumulated with the float offsets ca / cb; ours used exact references
-        Za *= exp2(static_cast<double>(ca) + static_cast<double>(pd.Ma) * kLog2eD);
-        Zb *= exp2(static_cast<double>(cb) + static_cast<double>(pd.Mb) * kLog2eD);
-    }
-    pp.item_bits[item] = accept_bit(pp, item, pd.finite != 0, D, a_row, b_row, dt, pd.Ma, ca, Za, pd.Mb, cb, Zb);
-    pp.item_status[item] = pd.finite ? 0 : FSD_ROW_NONFINITE;
-}
 
 template <int DT, int DIV>
 __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(StreamParams P) {
@@ -189,7 +186,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     constexpr int NT = (kTmemPerThread / EPT) < kMaxStagesPerPair ? (kTmemPerThread / EPT) : kMaxStagesPerPair;
     constexpr int NR = kMaxStagesPerPair - NT;       // stages kept in registers
     constexpr bool kSecondSweep = DIV != FSD_DIV_KL;
-    constexpr float kYMin = -150.f;                  // ex2 flushes to zero below -126
+    constexpr float kClamp = -1.0e30f;               // -inf logits are read as this: 2^y = 0 and 0 * y = 0 stay finite
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -200,7 +197,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     const int rank = static_cast<int>(cluster.block_rank());
     const int cluster_id = blockIdx.x / C, n_clusters = gridDim.x / C;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const PairParams& pp = P.pp;
 
     // this CTA's slice of every row, in vectors
     const int base = P.nvec_row / C, rem = P.nvec_row % C;
@@ -213,7 +209,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     if (blockIdx.x == 0 && tid == 0) *P.timeout_flag = 0;   // a wait needs far longer to run out than this store takes
     if (tid == 0) {
         for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kStreamWarps); }
-        sh.pend.item = -1;
+        sh.p_item = cluster_id; sh.p_stage = 0; sh.p_g = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -228,28 +224,28 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     const uint32_t taddr = sh.tmem_base + (static_cast<uint32_t>(32 * (warp & 3)) << 16) + static_cast<uint32_t>(64 * (warp >> 2));
 
     bool dead = false;                               // a bounded wait of this thread ran out
-    // ---- producer state (thread 0 only) ----
-    int p_item = cluster_id, p_stage = 0;
-    uint32_t p_g = 0;                                // stages issued so far
+
+    // ---- producer (thread 0 only) ----
+    // Rows of a pair; false for a tree node whose parent index is invalid (no data is moved for it).
     auto item_rows = [&](int item, const char*& a_row, const char*& b_row) -> bool {
-        const int b = item / pp.G, i = item - b * pp.G;
+        const int b = item / P.G, i = item - b * P.G;
         int trow = i;
-        if (pp.parent != nullptr) {
-            const int par = __ldg(pp.parent + item);
+        if (P.parent != nullptr) {
+            const int par = __ldg(P.parent + item);
             if (par < -1 || par >= i) return false;
             trow = par + 1;
         }
-        a_row = static_cast<const char*>(pp.target) + (static_cast<size_t>(b) * (pp.G + 1) + trow) * row_bytes;
-        b_row = static_cast<const char*>(pp.draft) + (static_cast<size_t>(b) * pp.G + i) * row_bytes;
+        a_row = static_cast<const char*>(P.target) + (static_cast<size_t>(b) * (P.G + 1) + trow) * row_bytes;
+        b_row = static_cast<const char*>(P.draft) + (static_cast<size_t>(b) * P.G + i) * row_bytes;
         return true;
     };
-    // issues the next stage if its ring slot is free (or, when `block`, waits for it); false if nothing was issued
+    // Issues the next stage if its ring slot is free (or, when `block`, waits for it); false if nothing was issued.
     auto produce = [&](bool block) -> bool {
-        while (p_item < P.n_items) {
-            const char *a_row, *b_row;
-            if (p_stage == 0 && !item_rows(p_item, a_row, b_row)) { p_item += n_clusters; continue; }   // bad tree node: no data
-            break;
-        }
+        int p_item = sh.p_item, p_stage = sh.p_stage;
+        const uint32_t p_g = sh.p_g;
+        const char *a_row = nullptr, *b_row = nullptr;
+        while (p_item < P.n_items && !item_rows(p_item, a_row, b_row)) p_item += n_clusters;
+        sh.p_item = p_item;
         if (p_item >= P.n_items) return false;
         const uint32_t slot = p_g % kRing;
         if (p_g >= kRing) {
@@ -257,8 +253,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
             if (block) mbar_wait(&sh.empty[slot], parity, P.timeout_flag, dead);
             else if (!mbar_try_wait(&sh.empty[slot], parity)) return false;
         }
-        const char *a_row, *b_row;
-        item_rows(p_item, a_row, b_row);
         const int v0 = p_stage * kStreamThreads;
         const int nv = (vcnt - v0) < kStreamThreads ? (vcnt - v0) : kStreamThreads;
         const uint32_t bytes = static_cast<uint32_t>(nv) * 16;
@@ -266,34 +260,37 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         mbar_arrive_expect_tx(&sh.full[slot], 2 * bytes);
         bulk_g2s(dst, a_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
         bulk_g2s(dst + kStageRowBytes, b_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
-        ++p_g;
+        sh.p_g = p_g + 1;
         if (++p_stage == ns) { p_stage = 0; p_item += n_clusters; }
+        sh.p_item = p_item; sh.p_stage = p_stage;
         return true;
     };
-    if (tid == 0) { while (p_g < kRing && produce(false)) {} }
+    if (tid == 0) { while (sh.p_g < kRing && produce(false)) {} }
+    __syncwarp();
 
     float ereg[(NR > 0 ? NR : 1) * EPT];
     uint32_t g = 0;                                  // stages consumed so far
     int parity = 0;                                  // exchange slot parity
-    float x_carry = 0.f;                             // this thread's share of the previous pair's second-sweep sum (warp-reduced, lane 0)
-    bool have_prev = false;
+    float x_carry = 0.f;                             // previous pair's second-sweep sum of this warp
+    int prev_item = -1;                              // pair whose second-sweep sum is still to be published
 
     for (int item = cluster_id;; item += n_clusters) {
-        const bool live = item < P.n_items;          // one extra round flushes the last pair's second sweep
-        if (!live && !have_prev) break;
+        const bool live = item < P.n_items;          // one extra round publishes the last pair's second sweep
+        if (!live && prev_item < 0) break;
         bool bad = false;
-        if (live && pp.parent != nullptr) {
-            const int i = item % pp.G;
-            const int par = __ldg(pp.parent + item);
+        if (live && P.parent != nullptr) {
+            const int i = item % P.G;
+            const int par = __ldg(P.parent + item);
             bad = par < -1 || par >= i;
         }
         const bool work = live && !bad;
 
-        float ra = -INFINITY, rb = -INFINITY, za = 0.f, zb = 0.f, sa = 0.f, sb = 0.f, kk = 0.f;
-        uint32_t diff = 0;
+        float ka = -INFINITY, kb = -INFINITY;
         if (work) {
+            float ra = -INFINITY, rb = -INFINITY, za = 0.f, zb = 0.f, sa = 0.f, sb = 0.f, kk = 0.f;
+            uint32_t diff = 0;
             // ---- sweep A: exact thread maxima and the bitwise difference flag, from shared memory ----
-            if (tid == 0) { while (p_g < g + ns && produce(true)) {} }
+            if (tid == 0) { while (sh.p_g < g + ns && produce(true)) {} }
             __syncwarp();
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
@@ -306,8 +303,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                         const uint4 vb = *reinterpret_cast<const uint4*>(st + kStageRowBytes);
                         diff |= (va.x ^ vb.x) | (va.y ^ vb.y) | (va.z ^ vb.z) | (va.w ^ vb.w);
                         if constexpr (DT == FSD_BF16) {
-                            const uint32_t ma = bf16x2_max(bf16x2_max(va.x, va.y), bf16x2_max(va.z, va.w));
-                            const uint32_t mb = bf16x2_max(bf16x2_max(vb.x, vb.y), bf16x2_max(vb.z, vb.w));
+                            const uint32_t ma = bf16x2_max_nan(bf16x2_max_nan(va.x, va.y), bf16x2_max_nan(va.z, va.w));
+                            const uint32_t mb = bf16x2_max_nan(bf16x2_max_nan(vb.x, vb.y), bf16x2_max_nan(vb.z, vb.w));
                             ra = fmax_nan(ra, fmax_nan(bf16_lo(ma), bf16_hi(ma)));
                             rb = fmax_nan(rb, fmax_nan(bf16_lo(mb), bf16_hi(mb)));
                         } else {
@@ -319,9 +316,12 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                     }
                 }
             }
+            // integer references in the log2 domain: y = logit*log2e - k <= 0 up to rounding
+            ka = ra == -INFINITY ? -INFINITY : ceilf(ra * kLog2e);
+            kb = rb == -INFINITY ? -INFINITY : ceilf(rb * kLog2e);
+            const float ca = ra == -INFINITY ? 0.f : -ka, cb = rb == -INFINITY ? 0.f : -kb;
+
             // ---- sweep B: exponentials, sums, park the e values ----
-            const float ca = ra == -INFINITY ? 0.f : -ra * kLog2e;
-            const float cb = rb == -INFINITY ? 0.f : -rb * kLog2e;
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
                 if (s < ns) {
@@ -329,13 +329,28 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                     float e[EPT];
                     if (s * kStreamThreads + tid < vcnt) {
                         const unsigned char* st = ring + slot * kStageBytes + tid * 16;
+                        uint4 va = *reinterpret_cast<const uint4*>(st);
+                        uint4 vb = *reinterpret_cast<const uint4*>(st + kStageRowBytes);
                         float xa[EPV], xb[EPV];
-                        unpack_vec<DT>(*reinterpret_cast<const uint4*>(st), xa);
-                        unpack_vec<DT>(*reinterpret_cast<const uint4*>(st + kStageRowBytes), xb);
+                        if constexpr (DT == FSD_BF16) {
+                            constexpr uint32_t kClamp2 = 0xF149F149u;     // bf16x2 (-1e30, -1e30)
+                            va.x = bf16x2_max(va.x, kClamp2); va.y = bf16x2_max(va.y, kClamp2);
+                            va.z = bf16x2_max(va.z, kClamp2); va.w = bf16x2_max(va.w, kClamp2);
+                            if constexpr (DIV != FSD_DIV_KL) {            // KL needs the draft's -inf: q = 0 < p gives +inf
+                                vb.x = bf16x2_max(vb.x, kClamp2); vb.y = bf16x2_max(vb.y, kClamp2);
+                                vb.z = bf16x2_max(vb.z, kClamp2); vb.w = bf16x2_max(vb.w, kClamp2);
+                            }
+                        }
+                        unpack_vec<DT>(va, xa);
+                        unpack_vec<DT>(vb, xb);
 #pragma unroll
                         for (int j = 0; j < EPV; ++j) {
-                            const float ya_raw = fmaf(xa[j], kLog2e, ca), yb_raw = fmaf(xb[j], kLog2e, cb);
-                            const float ya = fmaxf(ya_raw, kYMin), yb = fmaxf(yb_raw, kYMin);
+                            float av = xa[j], bv = xb[j];
+                            if constexpr (DT == FSD_F32) {
+                                av = fmaxf(av, kClamp);
+                                if constexpr (DIV != FSD_DIV_KL) bv = fmaxf(bv, kClamp);
+                            }
+                            const float ya = fmaf(av, kLog2e, ca), yb = fmaf(bv, kLog2e, cb);
                             const float ea = ex2(ya), eb = ex2(yb);
                             za += ea;
                             zb += eb;
@@ -344,8 +359,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                                 sb = fmaf(eb, yb, sb);
                             }
                             if constexpr (DIV == FSD_DIV_KL) {
-                                // q = 0 < p must give +inf: the draft exponent is used unclamped
-                                if (ea > 0.f) kk = fmaf(ea, ya - yb_raw, kk);
+                                if (ea > 0.f) kk = fmaf(ea, ya - yb, kk);
                             }
                             e[j] = ea;
                             e[EPV + j] = eb;
@@ -365,17 +379,15 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                     // this warp is done with the slot
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sh.empty[slot]);
-                    if (tid == 0) produce(false);
-                    __syncwarp();
                 }
             }
             g += ns;
             if constexpr (kSecondSweep) tmem_wait_st();
 
-            // ---- thread -> warp: bring the sums to the warp's reference ----
-            const float wa = warp_max_nan(ra), wb = warp_max_nan(rb);
-            const float da = ra == -INFINITY ? 0.f : (ra - wa) * kLog2e, db = rb == -INFINITY ? 0.f : (rb - wb) * kLog2e;
-            const float fa = ra == -INFINITY ? 0.f : ex2(da), fb = rb == -INFINITY ? 0.f : ex2(db);
+            // ---- thread -> warp: bring the sums to the warp's reference (exact power-of-two factors) ----
+            const float wka = warp_max_nan(ka), wkb = warp_max_nan(kb);
+            const float da = ka == -INFINITY ? 0.f : ka - wka, db = kb == -INFINITY ? 0.f : kb - wkb;
+            const float fa = ka == -INFINITY ? 0.f : pow2_int(da), fb = kb == -INFINITY ? 0.f : pow2_int(db);
             float v_za = za * fa, v_zb = zb * fb;
             float v_sa = fa * fmaf(da, za, sa), v_sb = fb * fmaf(db, zb, sb);
             float v_kk = fa * fmaf(da - db, za, kk);
@@ -392,98 +404,98 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
             const uint32_t wdiff = __reduce_or_sync(0xffffffffu, diff);
             if (lane == 0) {
                 WarpStats& w = sh.ws[warp];
-                w.ra = wa; w.rb = wb; w.za = v_za; w.zb = v_zb; w.sa = v_sa; w.sb = v_sb; w.kk = v_kk; w.diff = wdiff;
+                w.ka = wka; w.kb = wkb; w.za = v_za; w.zb = v_zb; w.sa = v_sa; w.sb = v_sb; w.kk = v_kk; w.diff = wdiff;
             }
+        } else if (lane == 0) {
+            WarpStats& w = sh.ws[warp];
+            w.ka = -INFINITY; w.kb = -INFINITY; w.za = 0.f; w.zb = 0.f; w.sa = 0.f; w.sb = 0.f; w.kk = 0.f; w.diff = 0;
         }
-        if (lane == 0) sh.wx[warp] = x_carry;         // previous pair's second-sweep sum of this warp
-        __syncthreads();                               // (A) warp statistics visible
+        if (lane == 0) sh.ws[warp].x = x_carry;
+        __syncthreads();                               // warp statistics visible in the CTA
 
-        // ---- warp 0: CTA totals, publish to the cluster ----
-        if (warp == 0) {
-            double Za = 0, Zb = 0, Sa = 0, Sb = 0, K = 0, X = 0;
-            float Ra = -INFINITY, Rb = -INFINITY;
-            uint32_t df = 0;
+        // ---- every warp: CTA totals (each lane < 16 takes one warp's entry) ----
+        float Ka, Kb;
+        uint32_t DF;
+        {
+            float eka = -INFINITY, ekb = -INFINITY, eza = 0.f, ezb = 0.f, esa = 0.f, esb = 0.f, ekk = 0.f, ex = 0.f;
+            uint32_t edf = 0;
             if (lane < kStreamWarps) {
-                X = static_cast<double>(sh.wx[lane]);
-                if (work) {
-                    const WarpStats w = sh.ws[lane];
-                    Ra = w.ra; Rb = w.rb; df = w.diff;
-                    Za = w.za; Zb = w.zb; Sa = w.sa; Sb = w.sb; K = w.kk;
-                }
+                const WarpStats w = sh.ws[lane];
+                eka = w.ka; ekb = w.kb; eza = w.za; ezb = w.zb; esa = w.sa; esb = w.sb; ekk = w.kk; ex = w.x; edf = w.diff;
             }
-            const float cRa = warp_max_nan(Ra), cRb = warp_max_nan(Rb);
-            // rescale each warp's sums to the CTA reference (double; -inf references carry zero sums)
-            const double da = (Ra == -INFINITY) ? 0.0 : (static_cast<double>(Ra) - cRa) * kLog2eD;
-            const double db = (Rb == -INFINITY) ? 0.0 : (static_cast<double>(Rb) - cRb) * kLog2eD;
-            const double fa = (Ra == -INFINITY) ? 0.0 : exp2(da), fb = (Rb == -INFINITY) ? 0.0 : exp2(db);
-            K = fa * (K + (da - db) * Za);
-            Sa = fa * (Sa + da * Za); Sb = fb * (Sb + db * Zb);
-            Za *= fa; Zb *= fb;
-            Za = warp_sum(Za); Zb = warp_sum(Zb); Sa = warp_sum(Sa); Sb = warp_sum(Sb); K = warp_sum(K); X = warp_sum(X);
-            df = __reduce_or_sync(0xffffffffu, df);
-            if (lane == 0) {
+            Ka = warp_max_nan(eka); Kb = warp_max_nan(ekb);
+            const float da = eka == -INFINITY ? 0.f : eka - Ka, db = ekb == -INFINITY ? 0.f : ekb - Kb;
+            const float fa = eka == -INFINITY ? 0.f : pow2_int(da), fb = ekb == -INFINITY ? 0.f : pow2_int(db);
+            float Za = eza * fa, Zb = ezb * fb;
+            float Sa = fa * fmaf(da, eza, esa), Sb = fb * fmaf(db, ezb, esb);
+            float KK = fa * fmaf(da - db, eza, ekk);
+            float X = ex;
+#pragma unroll
+            for (int m = 8; m > 0; m >>= 1) {
+                Za += __shfl_xor_sync(0xffffffffu, Za, m); Zb += __shfl_xor_sync(0xffffffffu, Zb, m);
+                Sa += __shfl_xor_sync(0xffffffffu, Sa, m); Sb += __shfl_xor_sync(0xffffffffu, Sb, m);
+                KK += __shfl_xor_sync(0xffffffffu, KK, m); X += __shfl_xor_sync(0xffffffffu, X, m);
+            }
+            DF = __reduce_or_sync(0xffffffffu, edf);
+            if (tid == 0) {
                 CtaStats& c = sh.xch[parity];
-                c.ra = cRa; c.rb = cRb; c.za = Za; c.zb = Zb; c.sa = Sa; c.sb = Sb; c.kk = K; c.x_prev = X; c.diff = df;
+                c.ka = Ka; c.kb = Kb; c.za = Za; c.zb = Zb; c.sa = Sa; c.sb = Sb; c.kk = KK; c.x = X; c.diff = DF;
             }
         }
-        cluster.sync();                                // every CTA's statistics visible cluster-wide
+        cluster.sync();                                // every CTA's totals visible cluster-wide
 
-        // ---- warp 0: cluster totals; broadcast what the second sweep needs; queue the finish ----
-        if (warp == 0) {
-            double Za = 0, Zb = 0, Sa = 0, Sb = 0, K = 0, X = 0;
-            float Ra = -INFINITY, Rb = -INFINITY;
-            uint32_t df = 0;
+        // ---- every warp: cluster totals in double (each lane < C takes one CTA's entry) ----
+        double tZa, tZb, tSa, tSb, tK, tX;
+        {
+            float eka = -INFINITY, ekb = -INFINITY;
+            double eza = 0, ezb = 0, esa = 0, esb = 0, ekk = 0, ex = 0;
+            uint32_t edf = 0;
             if (lane < C) {
                 const CtaStats* c = &cluster.map_shared_rank(&sh, lane)->xch[parity];
-                Ra = c->ra; Rb = c->rb; Za = c->za; Zb = c->zb; Sa = c->sa; Sb = c->sb; K = c->kk; X = c->x_prev; df = c->diff;
+                eka = c->ka; ekb = c->kb; eza = c->za; ezb = c->zb; esa = c->sa; esb = c->sb; ekk = c->kk; ex = c->x; edf = c->diff;
             }
-            const float Ma = warp_max_nan(Ra), Mb = warp_max_nan(Rb);
-            const double da = (Ra == -INFINITY) ? 0.0 : (static_cast<double>(Ra) - Ma) * kLog2eD;
-            const double db = (Rb == -INFINITY) ? 0.0 : (static_cast<double>(Rb) - Mb) * kLog2eD;
-            const double fa = (Ra == -INFINITY) ? 0.0 : exp2(da), fb = (Rb == -INFINITY) ? 0.0 : exp2(db);
-            K = fa * (K + (da - db) * Za);
-            Sa = fa * (Sa + da * Za); Sb = fb * (Sb + db * Zb);
-            Za *= fa; Zb *= fb;
-            Za = warp_sum(Za); Zb = warp_sum(Zb); Sa = warp_sum(Sa); Sb = warp_sum(Sb); K = warp_sum(K); X = warp_sum(X);
-            df = __reduce_or_sync(0xffffffffu, df);
-            if (lane == 0) {
-                // finish the previous pair now that its second-sweep sum is complete (rank 0 only)
-                if (rank == 0 && sh.pend.item >= 0) {
-                    finish_pair(P, sh.pend, X, DT);
-                    sh.pend.item = -1;
-                }
-                if (live) {
-                    const bool finite = work && isfinite(Ma) && isfinite(Mb) && isfinite(Za) && isfinite(Zb) && Za > 0.0 && Zb > 0.0;
-                    sh.bc_Ma = Ma; sh.bc_Mb = Mb;
-                    sh.bc_iZa = finite ? static_cast<float>(1.0 / Za) : 0.f;
-                    sh.bc_iZb = finite ? static_cast<float>(1.0 / Zb) : 0.f;
-                    if (rank == 0) {
-                        Pending& pd = sh.pend;
-                        if (bad) {
-                            pp.divergence[item] = __int_as_float(0x7fc00000);
-                            pp.item_bits[item] = 0;
-                            pp.item_status[item] = FSD_ROW_BADTREE;
-                        } else {
-                            pd.item = item; pd.finite = finite; pd.differ = df != 0;
-                            pd.Ma = Ma; pd.Mb = Mb; pd.Za = Za; pd.Zb = Zb; pd.Sa = Sa; pd.Sb = Sb; pd.K = K;
-                        }
-                    }
-                }
+            Ka = warp_max_nan(eka); Kb = warp_max_nan(ekb);
+            const float da = eka == -INFINITY ? 0.f : eka - Ka, db = ekb == -INFINITY ? 0.f : ekb - Kb;
+            const double fa = eka == -INFINITY ? 0.0 : static_cast<double>(pow2_int(da));
+            const double fb = ekb == -INFINITY ? 0.0 : static_cast<double>(pow2_int(db));
+            tK = fa * (ekk + static_cast<double>(da - db) * eza);
+            tSa = fa * (esa + static_cast<double>(da) * eza); tSb = fb * (esb + static_cast<double>(db) * ezb);
+            tZa = eza * fa; tZb = ezb * fb;
+            tX = ex;
+#pragma unroll
+            for (int m = 4; m > 0; m >>= 1) {
+                tZa += shfl_xor_d(tZa, m); tZb += shfl_xor_d(tZb, m); tSa += shfl_xor_d(tSa, m);
+                tSb += shfl_xor_d(tSb, m); tK += shfl_xor_d(tK, m); tX += shfl_xor_d(tX, m);
+            }
+            DF = __reduce_or_sync(0xffffffffu, edf);
+            // the sums live in lanes 0..7; every lane needs the two normalisers for the second sweep
+            tZa = __shfl_sync(0xffffffffu, tZa, 0);
+            tZb = __shfl_sync(0xffffffffu, tZb, 0);
+        }
+        // ---- rank 0 records the totals; the previous pair gets its second-sweep sum ----
+        if (rank == 0 && tid == kStreamThreads - 32) {
+            if (prev_item >= 0) P.records[prev_item].X = tX;
+            if (live) {
+                PairRecord r;
+                r.Za = tZa; r.Zb = tZb; r.Sa = tSa; r.Sb = tSb; r.K = tK; r.X = 0.0;
+                r.ka = Ka; r.kb = Kb; r.differ = DF; r.state = bad ? kRecordBadTree : kRecordStats;
+                P.records[item] = r;
             }
         }
-        __syncthreads();                               // (B) broadcast visible
         if (tid == 0) { while (produce(false)) {} }
         __syncwarp();
         parity ^= 1;
-        have_prev = false;
+        prev_item = -1;
         x_carry = 0.f;
         if (!live) break;
+        prev_item = item;
 
         // ---- second sweep over the parked e values ----
         if (work && kSecondSweep) {
-            const float Ma = sh.bc_Ma, Mb = sh.bc_Mb;
-            const float ia = ra == -INFINITY ? 0.f : ex2((ra - Ma) * kLog2e) * sh.bc_iZa;
-            const float ib = rb == -INFINITY ? 0.f : ex2((rb - Mb) * kLog2e) * sh.bc_iZb;
+            const bool ok = tZa > 0.0 && tZb > 0.0 && tZa < 3.0e38 && tZb < 3.0e38;     // false for NaN too
+            const float iza = ok ? 1.0f / static_cast<float>(tZa) : 0.f, izb = ok ? 1.0f / static_cast<float>(tZb) : 0.f;
+            const float ia = (ka == -INFINITY || !ok) ? 0.f : pow2_int(ka - Ka) * iza;
+            const float ib = (kb == -INFINITY || !ok) ? 0.f : pow2_int(kb - Kb) * izb;
             float x = 0.f;
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
@@ -496,8 +508,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
 #pragma unroll
                         for (int j = 0; j < EPT; ++j) e[j] = ereg[(s - NT < 0 ? 0 : s - NT) * EPT + j];
                     }
-                    if (tid == 0) produce(false);
-                    __syncwarp();
 #pragma unroll
                     for (int j = 0; j < EPV; ++j) {
                         if constexpr (DIV == FSD_DIV_JS) {
@@ -513,7 +523,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
             for (int m = 16; m > 0; m >>= 1) x += __shfl_xor_sync(0xffffffffu, x, m);
             x_carry = x;
         }
-        have_prev = true;
     }
 
     // ---- release tensor memory ----
@@ -523,6 +532,16 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sh.tmem_base), "r"(kTmemCols) : "memory");
     }
     cluster.sync();                                    // nobody leaves while a peer may still read its shared memory
+}
+
+// Occupancy twin: same block size, register bound and dynamic shared memory as the streaming
+// kernel but no tensor-memory instructions.  The occupancy calculator assumes one resident CTA
+// per SM for any kernel that allocates tensor memory (it cannot know how many columns); the
+// streaming kernel allocates half of an SM's tensor memory, so two CTAs do fit, and the grid
+// is sized from this twin instead.
+__global__ void __launch_bounds__(kStreamThreads, 2) fsd_stream_occupancy_twin(int* p) {
+    extern __shared__ unsigned char smem_raw[];
+    if (p != nullptr) p[threadIdx.x] = smem_raw[threadIdx.x];
 }
 
 }  // namespace fsd
