@@ -169,11 +169,8 @@ struct CtaStats {              // one per CTA and parity, read by the whole clus
 };
 struct StreamShared {
     uint64_t full[kRing];
-    uint64_t empty[kRing];
+    int readers_done[kRing];   // warps that have finished reading the slot's current stage
     uint32_t tmem_base;
-    // producer cursor (thread 0 only; kept here to spare registers)
-    int p_item, p_stage;
-    uint32_t p_g;
     WarpStats ws[kStreamWarps];
     CtaStats xch[2];
 };
@@ -208,8 +205,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     // ---- set-up: barriers, tensor memory ----
     if (blockIdx.x == 0 && tid == 0) *P.timeout_flag = 0;   // a wait needs far longer to run out than this store takes
     if (tid == 0) {
-        for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kStreamWarps); }
-        sh.p_item = cluster_id; sh.p_stage = 0; sh.p_g = 0;
+        for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); sh.readers_done[s] = 0; }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -225,47 +221,35 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
 
     bool dead = false;                               // a bounded wait of this thread ran out
 
-    // ---- producer (thread 0 only) ----
-    // Rows of a pair; false for a tree node whose parent index is invalid (no data is moved for it).
-    auto item_rows = [&](int item, const char*& a_row, const char*& b_row) -> bool {
-        const int b = item / P.G, i = item - b * P.G;
+    // ---- producer: stage number -> (pair, slice part); any thread may issue a stage ----
+    // Stage gg of this CTA is part gg % ns of the (gg / ns)-th pair of this cluster.  The warp
+    // that is last to finish reading a ring slot refills it at once (see sweep B), so the
+    // copies are issued as early as possible and the work is spread over the warps.
+    auto issue_stage = [&](uint32_t gg) {
+        const uint32_t k = gg / static_cast<uint32_t>(ns), s = gg - k * static_cast<uint32_t>(ns);
+        const long long item = cluster_id + static_cast<long long>(k) * n_clusters;
+        if (item >= P.n_items) return;
+        const int b = static_cast<int>(item / P.G), i = static_cast<int>(item - static_cast<long long>(b) * P.G);
         int trow = i;
         if (P.parent != nullptr) {
             const int par = __ldg(P.parent + item);
-            if (par < -1 || par >= i) return false;
-            trow = par + 1;
+            trow = (par >= -1 && par < i) ? par + 1 : 0;       // an invalid node still moves (ignored) data
         }
-        a_row = static_cast<const char*>(P.target) + (static_cast<size_t>(b) * (P.G + 1) + trow) * row_bytes;
-        b_row = static_cast<const char*>(P.draft) + (static_cast<size_t>(b) * P.G + i) * row_bytes;
-        return true;
-    };
-    // Issues the next stage if its ring slot is free (or, when `block`, waits for it); false if nothing was issued.
-    auto produce = [&](bool block) -> bool {
-        int p_item = sh.p_item, p_stage = sh.p_stage;
-        const uint32_t p_g = sh.p_g;
-        const char *a_row = nullptr, *b_row = nullptr;
-        while (p_item < P.n_items && !item_rows(p_item, a_row, b_row)) p_item += n_clusters;
-        sh.p_item = p_item;
-        if (p_item >= P.n_items) return false;
-        const uint32_t slot = p_g % kRing;
-        if (p_g >= kRing) {
-            const uint32_t parity = ((p_g / kRing) - 1) & 1;
-            if (block) mbar_wait(&sh.empty[slot], parity, P.timeout_flag, dead);
-            else if (!mbar_try_wait(&sh.empty[slot], parity)) return false;
-        }
-        const int v0 = p_stage * kStreamThreads;
+        const char* a_row = static_cast<const char*>(P.target) + (static_cast<size_t>(b) * (P.G + 1) + trow) * row_bytes;
+        const char* b_row = static_cast<const char*>(P.draft) + (static_cast<size_t>(b) * P.G + i) * row_bytes;
+        const uint32_t slot = gg % kRing;
+        const int v0 = static_cast<int>(s) * kStreamThreads;
         const int nv = (vcnt - v0) < kStreamThreads ? (vcnt - v0) : kStreamThreads;
         const uint32_t bytes = static_cast<uint32_t>(nv) * 16;
         unsigned char* dst = ring + slot * kStageBytes;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of the slot precede the async writes
         mbar_arrive_expect_tx(&sh.full[slot], 2 * bytes);
         bulk_g2s(dst, a_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
         bulk_g2s(dst + kStageRowBytes, b_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
-        sh.p_g = p_g + 1;
-        if (++p_stage == ns) { p_stage = 0; p_item += n_clusters; }
-        sh.p_item = p_item; sh.p_stage = p_stage;
-        return true;
     };
-    if (tid == 0) { while (sh.p_g < kRing && produce(false)) {} }
+    if (tid == 0) {
+        for (uint32_t gg = 0; gg < kRing; ++gg) issue_stage(gg);
+    }
     __syncwarp();
 
     float ereg[(NR > 0 ? NR : 1) * EPT];
@@ -283,15 +267,13 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
             const int par = __ldg(P.parent + item);
             bad = par < -1 || par >= i;
         }
-        const bool work = live && !bad;
+        const bool work = live;                      // an invalid tree node is processed too; its record says so
 
         float ka = -INFINITY, kb = -INFINITY;
         if (work) {
             float ra = -INFINITY, rb = -INFINITY, za = 0.f, zb = 0.f, sa = 0.f, sb = 0.f, kk = 0.f;
             uint32_t diff = 0;
             // ---- sweep A: exact thread maxima and the bitwise difference flag, from shared memory ----
-            if (tid == 0) { while (sh.p_g < g + ns && produce(true)) {} }
-            __syncwarp();
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
                 if (s < ns) {
@@ -376,9 +358,16 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                             for (int j = 0; j < EPT; ++j) ereg[(s - NT < 0 ? 0 : s - NT) * EPT + j] = e[j];
                         }
                     }
-                    // this warp is done with the slot
+                    // this warp is done with the slot; the last warp to say so refills it
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&sh.empty[slot]);
+                    if (lane == 0) {
+                        __threadfence_block();
+                        if (atomicAdd(&sh.readers_done[slot], 1) == kStreamWarps - 1) {
+                            sh.readers_done[slot] = 0;
+                            issue_stage(gs + kRing);
+                        }
+                    }
+                    __syncwarp();
                 }
             }
             g += ns;
@@ -413,10 +402,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         if (lane == 0) sh.ws[warp].x = x_carry;
         __syncthreads();                               // warp statistics visible in the CTA
 
-        // ---- every warp: CTA totals (each lane < 16 takes one warp's entry) ----
+        // ---- warp 0: CTA totals (each lane < 16 takes one warp's entry) ----
         float Ka, Kb;
-        uint32_t DF;
-        {
+        if (warp == 0) {
+            uint32_t DF;
             float eka = -INFINITY, ekb = -INFINITY, eza = 0.f, ezb = 0.f, esa = 0.f, esb = 0.f, ekk = 0.f, ex = 0.f;
             uint32_t edf = 0;
             if (lane < kStreamWarps) {
@@ -444,46 +433,52 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         }
         cluster.sync();                                // every CTA's totals visible cluster-wide
 
-        // ---- every warp: cluster totals in double (each lane < C takes one CTA's entry) ----
-        double tZa, tZb, tSa, tSb, tK, tX;
+        // ---- every warp: cluster references and normalisers (each lane < C takes one CTA's entry) ----
+        float tZa, tZb;
         {
-            float eka = -INFINITY, ekb = -INFINITY;
-            double eza = 0, ezb = 0, esa = 0, esb = 0, ekk = 0, ex = 0;
-            uint32_t edf = 0;
-            if (lane < C) {
-                const CtaStats* c = &cluster.map_shared_rank(&sh, lane)->xch[parity];
-                eka = c->ka; ekb = c->kb; eza = c->za; ezb = c->zb; esa = c->sa; esb = c->sb; ekk = c->kk; ex = c->x; edf = c->diff;
-            }
+            const CtaStats* c = &cluster.map_shared_rank(&sh, lane < C ? lane : 0)->xch[parity];
+            float eka = -INFINITY, ekb = -INFINITY, eza = 0.f, ezb = 0.f;
+            if (lane < C) { eka = c->ka; ekb = c->kb; eza = c->za; ezb = c->zb; }
             Ka = warp_max_nan(eka); Kb = warp_max_nan(ekb);
             const float da = eka == -INFINITY ? 0.f : eka - Ka, db = ekb == -INFINITY ? 0.f : ekb - Kb;
-            const double fa = eka == -INFINITY ? 0.0 : static_cast<double>(pow2_int(da));
-            const double fb = ekb == -INFINITY ? 0.0 : static_cast<double>(pow2_int(db));
-            tK = fa * (ekk + static_cast<double>(da - db) * eza);
-            tSa = fa * (esa + static_cast<double>(da) * eza); tSb = fb * (esb + static_cast<double>(db) * ezb);
+            const float fa = eka == -INFINITY ? 0.f : pow2_int(da), fb = ekb == -INFINITY ? 0.f : pow2_int(db);
             tZa = eza * fa; tZb = ezb * fb;
-            tX = ex;
 #pragma unroll
             for (int m = 4; m > 0; m >>= 1) {
-                tZa += shfl_xor_d(tZa, m); tZb += shfl_xor_d(tZb, m); tSa += shfl_xor_d(tSa, m);
-                tSb += shfl_xor_d(tSb, m); tK += shfl_xor_d(tK, m); tX += shfl_xor_d(tX, m);
+                tZa += __shfl_xor_sync(0xffffffffu, tZa, m); tZb += __shfl_xor_sync(0xffffffffu, tZb, m);
             }
-            DF = __reduce_or_sync(0xffffffffu, edf);
-            // the sums live in lanes 0..7; every lane needs the two normalisers for the second sweep
             tZa = __shfl_sync(0xffffffffu, tZa, 0);
             tZb = __shfl_sync(0xffffffffu, tZb, 0);
-        }
-        // ---- rank 0 records the totals; the previous pair gets its second-sweep sum ----
-        if (rank == 0 && tid == kStreamThreads - 32) {
-            if (prev_item >= 0) P.records[prev_item].X = tX;
-            if (live) {
-                PairRecord r;
-                r.Za = tZa; r.Zb = tZb; r.Sa = tSa; r.Sb = tSb; r.K = tK; r.X = 0.0;
-                r.ka = Ka; r.kb = Kb; r.differ = DF; r.state = bad ? kRecordBadTree : kRecordStats;
-                P.records[item] = r;
+            // ---- one warp of rank 0: all totals in double, into the pair's record; the previous
+            //      pair gets its second-sweep sum ----
+            if (rank == 0 && warp == kStreamWarps - 1) {
+                double dza = 0, dzb = 0, dsa = 0, dsb = 0, dkk = 0, dx = 0;
+                uint32_t edf = 0;
+                if (lane < C) {
+                    const double ffa = fa, ffb = fb;
+                    dza = static_cast<double>(eza) * ffa; dzb = static_cast<double>(ezb) * ffb;
+                    dsa = ffa * (static_cast<double>(c->sa) + static_cast<double>(da) * eza);
+                    dsb = ffb * (static_cast<double>(c->sb) + static_cast<double>(db) * ezb);
+                    dkk = ffa * (static_cast<double>(c->kk) + static_cast<double>(da - db) * eza);
+                    dx = c->x; edf = c->diff;
+                }
+#pragma unroll
+                for (int m = 4; m > 0; m >>= 1) {
+                    dza += shfl_xor_d(dza, m); dzb += shfl_xor_d(dzb, m); dsa += shfl_xor_d(dsa, m);
+                    dsb += shfl_xor_d(dsb, m); dkk += shfl_xor_d(dkk, m); dx += shfl_xor_d(dx, m);
+                }
+                edf = __reduce_or_sync(0xffffffffu, edf);
+                if (lane == 0) {
+                    if (prev_item >= 0) P.records[prev_item].X = dx;
+                    if (live) {
+                        PairRecord r;
+                        r.Za = dza; r.Zb = dzb; r.Sa = dsa; r.Sb = dsb; r.K = dkk; r.X = 0.0;
+                        r.ka = Ka; r.kb = Kb; r.differ = edf; r.state = bad ? kRecordBadTree : kRecordStats;
+                        P.records[item] = r;
+                    }
+                }
             }
         }
-        if (tid == 0) { while (produce(false)) {} }
-        __syncwarp();
         parity ^= 1;
         prev_item = -1;
         x_carry = 0.f;
@@ -492,8 +487,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
 
         // ---- second sweep over the parked e values ----
         if (work && kSecondSweep) {
-            const bool ok = tZa > 0.0 && tZb > 0.0 && tZa < 3.0e38 && tZb < 3.0e38;     // false for NaN too
-            const float iza = ok ? 1.0f / static_cast<float>(tZa) : 0.f, izb = ok ? 1.0f / static_cast<float>(tZb) : 0.f;
+            const bool ok = tZa > 0.f && tZb > 0.f && tZa < 3.0e38f && tZb < 3.0e38f;   // false for NaN too
+            const float iza = ok ? 1.0f / tZa : 0.f, izb = ok ? 1.0f / tZb : 0.f;
             const float ia = (ka == -INFINITY || !ok) ? 0.f : pow2_int(ka - Ka) * iza;
             const float ib = (kb == -INFINITY || !ok) ? 0.f : pow2_int(kb - Kb) * izb;
             float x = 0.f;
