@@ -88,6 +88,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // already marked invalid and the kernel only has to reach its end.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* timeout_flag, bool& dead) {
     if (dead) return false;
+#pragma unroll 1
     for (uint32_t i = 0; i < kSpinLimit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     atomicExch(timeout_flag, 1);
@@ -148,6 +149,36 @@ __device__ __forceinline__ float warp_max_nan(float v) {
     for (int m = 16; m > 0; m >>= 1) v = fmax_nan(v, __shfl_xor_sync(0xffffffffu, v, m));
     return v;
 }
+// ---- packed pairs of floats (one instruction works on two values) --------------------------
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float sum2(uint64_t v) {
+    float lo, hi;
+    unpack2(v, lo, hi);
+    return lo + hi;
+}
+
 // 2^d for an integer-valued d <= 0 (exact); 0 below the normal range and for d = -inf; NaN for NaN
 __device__ __forceinline__ float pow2_int(float d) {
     if (d != d) return d;
@@ -271,7 +302,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
 
         float ka = -INFINITY, kb = -INFINITY;
         if (work) {
-            float ra = -INFINITY, rb = -INFINITY, za = 0.f, zb = 0.f, sa = 0.f, sb = 0.f, kk = 0.f;
+            float ra = -INFINITY, rb = -INFINITY, kk = 0.f;
+            uint64_t za2 = 0, zb2 = 0, sa2 = 0, sb2 = 0;     // packed (even, odd) partial sums
             uint32_t diff = 0;
             // ---- sweep A: exact thread maxima and the bitwise difference flag, from shared memory ----
 #pragma unroll
@@ -325,26 +357,32 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                         }
                         unpack_vec<DT>(va, xa);
                         unpack_vec<DT>(vb, xb);
+                        const uint64_t l2 = pack2(kLog2e, kLog2e), ca2 = pack2(ca, ca), cb2 = pack2(cb, cb);
 #pragma unroll
-                        for (int j = 0; j < EPV; ++j) {
-                            float av = xa[j], bv = xb[j];
+                        for (int j = 0; j < EPV; j += 2) {
+                            float a0 = xa[j], a1 = xa[j + 1], b0 = xb[j], b1 = xb[j + 1];
                             if constexpr (DT == FSD_F32) {
-                                av = fmaxf(av, kClamp);
-                                if constexpr (DIV != FSD_DIV_KL) bv = fmaxf(bv, kClamp);
+                                a0 = fmaxf(a0, kClamp); a1 = fmaxf(a1, kClamp);
+                                if constexpr (DIV != FSD_DIV_KL) { b0 = fmaxf(b0, kClamp); b1 = fmaxf(b1, kClamp); }
                             }
-                            const float ya = fmaf(av, kLog2e, ca), yb = fmaf(bv, kLog2e, cb);
-                            const float ea = ex2(ya), eb = ex2(yb);
-                            za += ea;
-                            zb += eb;
+                            const uint64_t ya2 = fma2(pack2(a0, a1), l2, ca2), yb2 = fma2(pack2(b0, b1), l2, cb2);
+                            float ya0, ya1, yb0, yb1;
+                            unpack2(ya2, ya0, ya1);
+                            unpack2(yb2, yb0, yb1);
+                            const float ea0 = ex2(ya0), ea1 = ex2(ya1), eb0 = ex2(yb0), eb1 = ex2(yb1);
+                            const uint64_t ea2 = pack2(ea0, ea1), eb2 = pack2(eb0, eb1);
+                            za2 = add2(za2, ea2);
+                            zb2 = add2(zb2, eb2);
                             if constexpr (DIV == FSD_DIV_JS) {
-                                sa = fmaf(ea, ya, sa);
-                                sb = fmaf(eb, yb, sb);
+                                sa2 = fma2(ea2, ya2, sa2);
+                                sb2 = fma2(eb2, yb2, sb2);
                             }
                             if constexpr (DIV == FSD_DIV_KL) {
-                                if (ea > 0.f) kk = fmaf(ea, ya - yb, kk);
+                                if (ea0 > 0.f) kk = fmaf(ea0, ya0 - yb0, kk);
+                                if (ea1 > 0.f) kk = fmaf(ea1, ya1 - yb1, kk);
                             }
-                            e[j] = ea;
-                            e[EPV + j] = eb;
+                            e[j] = ea0; e[j + 1] = ea1;
+                            e[EPV + j] = eb0; e[EPV + j + 1] = eb1;
                         }
                     } else {
 #pragma unroll
@@ -373,6 +411,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
             g += ns;
             if constexpr (kSecondSweep) tmem_wait_st();
 
+            const float za = sum2(za2), zb = sum2(zb2), sa = sum2(sa2), sb = sum2(sb2);
             // ---- thread -> warp: bring the sums to the warp's reference (exact power-of-two factors) ----
             const float wka = warp_max_nan(ka), wkb = warp_max_nan(kb);
             const float da = ka == -INFINITY ? 0.f : ka - wka, db = kb == -INFINITY ? 0.f : kb - wkb;
@@ -491,7 +530,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
             const float iza = ok ? 1.0f / tZa : 0.f, izb = ok ? 1.0f / tZb : 0.f;
             const float ia = (ka == -INFINITY || !ok) ? 0.f : pow2_int(ka - Ka) * iza;
             const float ib = (kb == -INFINITY || !ok) ? 0.f : pow2_int(kb - Kb) * izb;
-            float x = 0.f;
+            uint64_t x2 = 0;
+            float xt = 0.f;
+            // s = p + q + 2e-37 keeps lg2 finite where both terms vanish; the shift is below one ulp of any s that matters
+            const uint64_t ia2 = pack2(ia, ia), ib2 = pack2(ib, ib), tiny2 = pack2(1e-37f, 1e-37f);
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
                 if (s < ns) {
@@ -504,16 +546,24 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                         for (int j = 0; j < EPT; ++j) e[j] = ereg[(s - NT < 0 ? 0 : s - NT) * EPT + j];
                     }
 #pragma unroll
-                    for (int j = 0; j < EPV; ++j) {
+                    for (int j = 0; j < EPV; j += 2) {
+                        const uint64_t ea2 = pack2(e[j], e[j + 1]), eb2 = pack2(e[EPV + j], e[EPV + j + 1]);
                         if constexpr (DIV == FSD_DIV_JS) {
-                            const float sm = fmaxf(fmaf(e[EPV + j], ib, e[j] * ia), 1e-37f);
-                            x = fmaf(sm, lg2(sm), x);
+                            const uint64_t s2 = fma2(eb2, ib2, fma2(ea2, ia2, tiny2));
+                            float s0, s1;
+                            unpack2(s2, s0, s1);
+                            x2 = fma2(s2, pack2(lg2(s0), lg2(s1)), x2);
                         } else {
-                            x += fabsf(__fmul_rn(e[j], ia) - __fmul_rn(e[EPV + j], ib));
+                            // separately rounded products: a fused p - q would make TV(p, p) != 0
+                            const uint64_t d2 = fma2(mul2(eb2, ib2), pack2(-1.f, -1.f), mul2(ea2, ia2));
+                            float d0, d1;
+                            unpack2(d2, d0, d1);
+                            xt += fabsf(d0) + fabsf(d1);
                         }
                     }
                 }
             }
+            float x = sum2(x2) + xt;
 #pragma unroll
             for (int m = 16; m > 0; m >>= 1) x += __shfl_xor_sync(0xffffffffu, x, m);
             x_carry = x;
