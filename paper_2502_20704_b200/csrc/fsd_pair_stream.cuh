@@ -185,25 +185,47 @@ __device__ __forceinline__ float pow2_int(float d) {
     return d < -126.f ? 0.f : __int_as_float((static_cast<int>(d) + 127) << 23);
 }
 
+// ---- cluster-scope mbarrier helpers (the statistics exchange) ------------------------------
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, int* timeout_flag, bool& dead) {
+    if (dead) return false;
+#pragma unroll 1
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+    atomicExch(timeout_flag, 1);
+    dead = true;
+    return false;
+}
+// arrive (release, cluster scope) on the same-named barrier of CTA `rank` of this cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint64_t* bar, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+
 // ---- shared-memory layout ---------------------------------------------------------------
-struct WarpStats {             // one per warp, written by lane 0 after the exponential sweep
-    float ka, kb;              // warp references
-    float za, zb, sa, sb, kk;  // sums relative to the warp references
+struct PartStats {             // statistics of a warp (in ws) or of a CTA (in xch)
+    float ka, kb;              // references
+    float za, zb, sa, sb, kk;  // sums relative to the references
     float x;                   // second-sweep sum of the PREVIOUS pair
     uint32_t diff;
 };
-struct CtaStats {              // one per CTA and parity, read by the whole cluster
-    float ka, kb;
-    float za, zb, sa, sb, kk;
-    float x;
-    uint32_t diff;
-};
 struct StreamShared {
-    uint64_t full[kRing];
+    uint64_t full[kRing];      // a ring stage has landed
+    uint64_t xbar[2];          // every CTA of the cluster has delivered its statistics (per parity)
     int readers_done[kRing];   // warps that have finished reading the slot's current stage
+    int stats_done[2];         // warps that have posted their statistics (per parity)
     uint32_t tmem_base;
-    WarpStats ws[kStreamWarps];
-    CtaStats xch[2];
+    PartStats ws[2][kStreamWarps];
+    PartStats xch[2][kMaxClusterSize];     // written by the peers (and by this CTA for its own rank)
 };
 constexpr size_t kStreamSmemBytes = kRing * kStageBytes + sizeof(StreamShared) + 128;
 
@@ -237,6 +259,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     if (blockIdx.x == 0 && tid == 0) *P.timeout_flag = 0;   // a wait needs far longer to run out than this store takes
     if (tid == 0) {
         for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); sh.readers_done[s] = 0; }
+        mbar_init(&sh.xbar[0], C); mbar_init(&sh.xbar[1], C);
+        sh.stats_done[0] = 0; sh.stats_done[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -245,7 +269,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    cluster.sync();                                  // barriers of every CTA exist before any peer arrives on them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     // warp w owns tensor-memory lanes 32*(w%4)..+31 and columns 64*(w/4)..+63
     const uint32_t taddr = sh.tmem_base + (static_cast<uint32_t>(32 * (warp & 3)) << 16) + static_cast<uint32_t>(64 * (warp >> 2));
@@ -283,59 +307,70 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     }
     __syncwarp();
 
-    float ereg[(NR > 0 ? NR : 1) * EPT];
-    uint32_t g = 0;                                  // stages consumed so far
-    int parity = 0;                                  // exchange slot parity
-    float x_carry = 0.f;                             // previous pair's second-sweep sum of this warp
-    int prev_item = -1;                              // pair whose second-sweep sum is still to be published
-
-    for (int item = cluster_id;; item += n_clusters) {
-        const bool live = item < P.n_items;          // one extra round publishes the last pair's second sweep
-        if (!live && prev_item < 0) break;
-        bool bad = false;
-        if (live && P.parent != nullptr) {
-            const int i = item % P.G;
-            const int par = __ldg(P.parent + item);
-            bad = par < -1 || par >= i;
-        }
-        const bool work = live;                      // an invalid tree node is processed too; its record says so
-
-        float ka = -INFINITY, kb = -INFINITY;
-        if (work) {
-            float ra = -INFINITY, rb = -INFINITY, kk = 0.f;
-            uint64_t za2 = 0, zb2 = 0, sa2 = 0, sb2 = 0;     // packed (even, odd) partial sums
-            uint32_t diff = 0;
-            // ---- sweep A: exact thread maxima and the bitwise difference flag, from shared memory ----
+    // ---- sweep A: exact thread maxima and the bitwise difference flag of the pair starting at stage gA ----
+    auto sweep_a = [&](uint32_t gA, float& ra, float& rb, uint32_t& diff) {
+        ra = -INFINITY; rb = -INFINITY; diff = 0;
 #pragma unroll
-            for (int s = 0; s < kMaxStagesPerPair; ++s) {
-                if (s < ns) {
-                    const uint32_t gs = g + s, slot = gs % kRing;
-                    mbar_wait(&sh.full[slot], (gs / kRing) & 1, P.timeout_flag, dead);
-                    if (s * kStreamThreads + tid < vcnt) {
-                        const unsigned char* st = ring + slot * kStageBytes + tid * 16;
-                        const uint4 va = *reinterpret_cast<const uint4*>(st);
-                        const uint4 vb = *reinterpret_cast<const uint4*>(st + kStageRowBytes);
-                        diff |= (va.x ^ vb.x) | (va.y ^ vb.y) | (va.z ^ vb.z) | (va.w ^ vb.w);
-                        if constexpr (DT == FSD_BF16) {
-                            const uint32_t ma = bf16x2_max_nan(bf16x2_max_nan(va.x, va.y), bf16x2_max_nan(va.z, va.w));
-                            const uint32_t mb = bf16x2_max_nan(bf16x2_max_nan(vb.x, vb.y), bf16x2_max_nan(vb.z, vb.w));
-                            ra = fmax_nan(ra, fmax_nan(bf16_lo(ma), bf16_hi(ma)));
-                            rb = fmax_nan(rb, fmax_nan(bf16_lo(mb), bf16_hi(mb)));
-                        } else {
-                            ra = fmax_nan(ra, fmax_nan(fmax_nan(__uint_as_float(va.x), __uint_as_float(va.y)),
-                                                       fmax_nan(__uint_as_float(va.z), __uint_as_float(va.w))));
-                            rb = fmax_nan(rb, fmax_nan(fmax_nan(__uint_as_float(vb.x), __uint_as_float(vb.y)),
-                                                       fmax_nan(__uint_as_float(vb.z), __uint_as_float(vb.w))));
-                        }
+        for (int s = 0; s < kMaxStagesPerPair; ++s) {
+            if (s < ns) {
+                const uint32_t gs = gA + s, slot = gs % kRing;
+                mbar_wait(&sh.full[slot], (gs / kRing) & 1, P.timeout_flag, dead);
+                if (s * kStreamThreads + tid < vcnt) {
+                    const unsigned char* st = ring + slot * kStageBytes + tid * 16;
+                    const uint4 va = *reinterpret_cast<const uint4*>(st);
+                    const uint4 vb = *reinterpret_cast<const uint4*>(st + kStageRowBytes);
+                    diff |= (va.x ^ vb.x) | (va.y ^ vb.y) | (va.z ^ vb.z) | (va.w ^ vb.w);
+                    if constexpr (DT == FSD_BF16) {
+                        const uint32_t ma = bf16x2_max_nan(bf16x2_max_nan(va.x, va.y), bf16x2_max_nan(va.z, va.w));
+                        const uint32_t mb = bf16x2_max_nan(bf16x2_max_nan(vb.x, vb.y), bf16x2_max_nan(vb.z, vb.w));
+                        ra = fmax_nan(ra, fmax_nan(bf16_lo(ma), bf16_hi(ma)));
+                        rb = fmax_nan(rb, fmax_nan(bf16_lo(mb), bf16_hi(mb)));
+                    } else {
+                        ra = fmax_nan(ra, fmax_nan(fmax_nan(__uint_as_float(va.x), __uint_as_float(va.y)),
+                                                   fmax_nan(__uint_as_float(va.z), __uint_as_float(va.w))));
+                        rb = fmax_nan(rb, fmax_nan(fmax_nan(__uint_as_float(vb.x), __uint_as_float(vb.y)),
+                                                   fmax_nan(__uint_as_float(vb.z), __uint_as_float(vb.w))));
                     }
                 }
             }
+        }
+    };
+
+    float ereg[(NR > 0 ? NR : 1) * EPT];
+    uint32_t g = 0;                                  // first ring stage of the current pair
+    uint32_t li = 0;                                 // pairs this cluster has finished
+    float x_carry = 0.f;                             // previous pair's second-sweep sum of this warp
+    int prev_item = -1;                              // pair whose second-sweep sum is still to be published
+    int item = cluster_id;
+    float ra = -INFINITY, rb = -INFINITY;
+    uint32_t diff = 0;
+    if (item < P.n_items) sweep_a(0, ra, rb, diff);
+
+    for (;;) {
+        const bool live = item < P.n_items;          // one extra round publishes the last pair's second sweep
+        if (!live && prev_item < 0) break;
+        const int par = static_cast<int>(li & 1);
+        const uint32_t xphase = (li >> 1) & 1;
+        bool bad = false;
+        if (live && P.parent != nullptr) {
+            const int i = item % P.G;
+            const int pr = __ldg(P.parent + item);
+            bad = pr < -1 || pr >= i;
+        }
+
+        // ---- sweep B: exponentials, sums, park the e values; then this warp's statistics ----
+        float ka = -INFINITY, kb = -INFINITY;
+        PartStats mine;
+        mine.ka = -INFINITY; mine.kb = -INFINITY; mine.za = 0.f; mine.zb = 0.f; mine.sa = 0.f; mine.sb = 0.f; mine.kk = 0.f;
+        mine.diff = 0;
+        if (live) {
+            float kk = 0.f;
+            uint64_t za2 = 0, zb2 = 0, sa2 = 0, sb2 = 0;     // packed (even, odd) partial sums
             // integer references in the log2 domain: y = logit*log2e - k <= 0 up to rounding
             ka = ra == -INFINITY ? -INFINITY : ceilf(ra * kLog2e);
             kb = rb == -INFINITY ? -INFINITY : ceilf(rb * kLog2e);
             const float ca = ra == -INFINITY ? 0.f : -ka, cb = rb == -INFINITY ? 0.f : -kb;
-
-            // ---- sweep B: exponentials, sums, park the e values ----
+            const uint64_t l2 = pack2(kLog2e, kLog2e), ca2 = pack2(ca, ca), cb2 = pack2(cb, cb);
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
                 if (s < ns) {
@@ -357,7 +392,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                         }
                         unpack_vec<DT>(va, xa);
                         unpack_vec<DT>(vb, xb);
-                        const uint64_t l2 = pack2(kLog2e, kLog2e), ca2 = pack2(ca, ca), cb2 = pack2(cb, cb);
 #pragma unroll
                         for (int j = 0; j < EPV; j += 2) {
                             float a0 = xa[j], a1 = xa[j + 1], b0 = xb[j], b1 = xb[j + 1];
@@ -408,11 +442,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                     __syncwarp();
                 }
             }
-            g += ns;
             if constexpr (kSecondSweep) tmem_wait_st();
 
+            // thread -> warp: bring the sums to the warp's reference (exact power-of-two factors)
             const float za = sum2(za2), zb = sum2(zb2), sa = sum2(sa2), sb = sum2(sb2);
-            // ---- thread -> warp: bring the sums to the warp's reference (exact power-of-two factors) ----
             const float wka = warp_max_nan(ka), wkb = warp_max_nan(kb);
             const float da = ka == -INFINITY ? 0.f : ka - wka, db = kb == -INFINITY ? 0.f : kb - wkb;
             const float fa = ka == -INFINITY ? 0.f : pow2_int(da), fb = kb == -INFINITY ? 0.f : pow2_int(db);
@@ -429,84 +462,89 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                 }
                 if constexpr (DIV == FSD_DIV_KL) v_kk += __shfl_xor_sync(0xffffffffu, v_kk, m);
             }
-            const uint32_t wdiff = __reduce_or_sync(0xffffffffu, diff);
-            if (lane == 0) {
-                WarpStats& w = sh.ws[warp];
-                w.ka = wka; w.kb = wkb; w.za = v_za; w.zb = v_zb; w.sa = v_sa; w.sb = v_sb; w.kk = v_kk; w.diff = wdiff;
-            }
-        } else if (lane == 0) {
-            WarpStats& w = sh.ws[warp];
-            w.ka = -INFINITY; w.kb = -INFINITY; w.za = 0.f; w.zb = 0.f; w.sa = 0.f; w.sb = 0.f; w.kk = 0.f; w.diff = 0;
+            mine.ka = wka; mine.kb = wkb; mine.za = v_za; mine.zb = v_zb; mine.sa = v_sa; mine.sb = v_sb; mine.kk = v_kk;
+            mine.diff = __reduce_or_sync(0xffffffffu, diff);
         }
-        if (lane == 0) sh.ws[warp].x = x_carry;
-        __syncthreads();                               // warp statistics visible in the CTA
+        mine.x = x_carry;
 
-        // ---- warp 0: CTA totals (each lane < 16 takes one warp's entry) ----
-        float Ka, Kb;
-        if (warp == 0) {
-            uint32_t DF;
-            float eka = -INFINITY, ekb = -INFINITY, eza = 0.f, ezb = 0.f, esa = 0.f, esb = 0.f, ekk = 0.f, ex = 0.f;
-            uint32_t edf = 0;
-            if (lane < kStreamWarps) {
-                const WarpStats w = sh.ws[lane];
-                eka = w.ka; ekb = w.kb; eza = w.za; ezb = w.zb; esa = w.sa; esb = w.sb; ekk = w.kk; ex = w.x; edf = w.diff;
-            }
-            Ka = warp_max_nan(eka); Kb = warp_max_nan(ekb);
-            const float da = eka == -INFINITY ? 0.f : eka - Ka, db = ekb == -INFINITY ? 0.f : ekb - Kb;
-            const float fa = eka == -INFINITY ? 0.f : pow2_int(da), fb = ekb == -INFINITY ? 0.f : pow2_int(db);
-            float Za = eza * fa, Zb = ezb * fb;
-            float Sa = fa * fmaf(da, eza, esa), Sb = fb * fmaf(db, ezb, esb);
-            float KK = fa * fmaf(da - db, eza, ekk);
-            float X = ex;
+        // ---- post the warp's statistics; the last warp of the CTA to do so combines them and
+        //      delivers the CTA's statistics to every CTA of the cluster (itself included) ----
+        int last = 0;
+        if (lane == 0) {
+            sh.ws[par][warp] = mine;
+            __threadfence_block();
+            last = atomicAdd(&sh.stats_done[par], 1) == kStreamWarps - 1;
+            if (last) sh.stats_done[par] = 0;
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            __threadfence_block();
+            PartStats w;
+            w.ka = -INFINITY; w.kb = -INFINITY; w.za = 0.f; w.zb = 0.f; w.sa = 0.f; w.sb = 0.f; w.kk = 0.f; w.x = 0.f; w.diff = 0;
+            if (lane < kStreamWarps) w = sh.ws[par][lane];
+            PartStats c;
+            c.ka = warp_max_nan(w.ka); c.kb = warp_max_nan(w.kb);
+            const float da = w.ka == -INFINITY ? 0.f : w.ka - c.ka, db = w.kb == -INFINITY ? 0.f : w.kb - c.kb;
+            const float fa = w.ka == -INFINITY ? 0.f : pow2_int(da), fb = w.kb == -INFINITY ? 0.f : pow2_int(db);
+            c.za = w.za * fa; c.zb = w.zb * fb;
+            c.sa = fa * fmaf(da, w.za, w.sa); c.sb = fb * fmaf(db, w.zb, w.sb);
+            c.kk = fa * fmaf(da - db, w.za, w.kk);
+            c.x = w.x;
 #pragma unroll
             for (int m = 8; m > 0; m >>= 1) {
-                Za += __shfl_xor_sync(0xffffffffu, Za, m); Zb += __shfl_xor_sync(0xffffffffu, Zb, m);
-                Sa += __shfl_xor_sync(0xffffffffu, Sa, m); Sb += __shfl_xor_sync(0xffffffffu, Sb, m);
-                KK += __shfl_xor_sync(0xffffffffu, KK, m); X += __shfl_xor_sync(0xffffffffu, X, m);
+                c.za += __shfl_xor_sync(0xffffffffu, c.za, m); c.zb += __shfl_xor_sync(0xffffffffu, c.zb, m);
+                c.sa += __shfl_xor_sync(0xffffffffu, c.sa, m); c.sb += __shfl_xor_sync(0xffffffffu, c.sb, m);
+                c.kk += __shfl_xor_sync(0xffffffffu, c.kk, m); c.x += __shfl_xor_sync(0xffffffffu, c.x, m);
             }
-            DF = __reduce_or_sync(0xffffffffu, edf);
-            if (tid == 0) {
-                CtaStats& c = sh.xch[parity];
-                c.ka = Ka; c.kb = Kb; c.za = Za; c.zb = Zb; c.sa = Sa; c.sb = Sb; c.kk = KK; c.x = X; c.diff = DF;
+            c.diff = __reduce_or_sync(0xffffffffu, w.diff);
+            if (lane < C) {                                // lanes 0..15 hold the totals; lane r serves CTA r
+                cluster.map_shared_rank(&sh, lane)->xch[par][rank] = c;
+                mbar_arrive_remote(&sh.xbar[par], static_cast<uint32_t>(lane));
             }
         }
-        cluster.sync();                                // every CTA's totals visible cluster-wide
+        __syncwarp();
 
-        // ---- every warp: cluster references and normalisers (each lane < C takes one CTA's entry) ----
-        float tZa, tZb;
+        // ---- meanwhile: sweep A of the next pair ----
+        const int next = item + n_clusters;
+        float ra_n = -INFINITY, rb_n = -INFINITY;
+        uint32_t diff_n = 0;
+        if (live && next < P.n_items) sweep_a(g + ns, ra_n, rb_n, diff_n);
+
+        // ---- cluster totals: every CTA's statistics have arrived in this CTA's shared memory ----
+        mbar_wait_cluster(&sh.xbar[par], xphase, P.timeout_flag, dead);
+        float Ka, Kb, tZa, tZb;
         {
-            const CtaStats* c = &cluster.map_shared_rank(&sh, lane < C ? lane : 0)->xch[parity];
-            float eka = -INFINITY, ekb = -INFINITY, eza = 0.f, ezb = 0.f;
-            if (lane < C) { eka = c->ka; ekb = c->kb; eza = c->za; ezb = c->zb; }
-            Ka = warp_max_nan(eka); Kb = warp_max_nan(ekb);
-            const float da = eka == -INFINITY ? 0.f : eka - Ka, db = ekb == -INFINITY ? 0.f : ekb - Kb;
-            const float fa = eka == -INFINITY ? 0.f : pow2_int(da), fb = ekb == -INFINITY ? 0.f : pow2_int(db);
-            tZa = eza * fa; tZb = ezb * fb;
+            PartStats c;
+            c.ka = -INFINITY; c.kb = -INFINITY; c.za = 0.f; c.zb = 0.f; c.sa = 0.f; c.sb = 0.f; c.kk = 0.f; c.x = 0.f; c.diff = 0;
+            if (lane < C) c = sh.xch[par][lane];
+            Ka = warp_max_nan(c.ka); Kb = warp_max_nan(c.kb);
+            const float da = c.ka == -INFINITY ? 0.f : c.ka - Ka, db = c.kb == -INFINITY ? 0.f : c.kb - Kb;
+            const float fa = c.ka == -INFINITY ? 0.f : pow2_int(da), fb = c.kb == -INFINITY ? 0.f : pow2_int(db);
+            tZa = c.za * fa; tZb = c.zb * fb;
 #pragma unroll
             for (int m = 4; m > 0; m >>= 1) {
                 tZa += __shfl_xor_sync(0xffffffffu, tZa, m); tZb += __shfl_xor_sync(0xffffffffu, tZb, m);
             }
             tZa = __shfl_sync(0xffffffffu, tZa, 0);
             tZb = __shfl_sync(0xffffffffu, tZb, 0);
-            // ---- one warp of rank 0: all totals in double, into the pair's record; the previous
-            //      pair gets its second-sweep sum ----
+            // one warp of rank 0: all totals in double, into the pair's record; the previous pair
+            // gets its second-sweep sum
             if (rank == 0 && warp == kStreamWarps - 1) {
                 double dza = 0, dzb = 0, dsa = 0, dsb = 0, dkk = 0, dx = 0;
-                uint32_t edf = 0;
                 if (lane < C) {
                     const double ffa = fa, ffb = fb;
-                    dza = static_cast<double>(eza) * ffa; dzb = static_cast<double>(ezb) * ffb;
-                    dsa = ffa * (static_cast<double>(c->sa) + static_cast<double>(da) * eza);
-                    dsb = ffb * (static_cast<double>(c->sb) + static_cast<double>(db) * ezb);
-                    dkk = ffa * (static_cast<double>(c->kk) + static_cast<double>(da - db) * eza);
-                    dx = c->x; edf = c->diff;
+                    dza = static_cast<double>(c.za) * ffa; dzb = static_cast<double>(c.zb) * ffb;
+                    dsa = ffa * (static_cast<double>(c.sa) + static_cast<double>(da) * c.za);
+                    dsb = ffb * (static_cast<double>(c.sb) + static_cast<double>(db) * c.zb);
+                    dkk = ffa * (static_cast<double>(c.kk) + static_cast<double>(da - db) * c.za);
+                    dx = c.x;
                 }
 #pragma unroll
                 for (int m = 4; m > 0; m >>= 1) {
                     dza += shfl_xor_d(dza, m); dzb += shfl_xor_d(dzb, m); dsa += shfl_xor_d(dsa, m);
                     dsb += shfl_xor_d(dsb, m); dkk += shfl_xor_d(dkk, m); dx += shfl_xor_d(dx, m);
                 }
-                edf = __reduce_or_sync(0xffffffffu, edf);
+                const uint32_t edf = __reduce_or_sync(0xffffffffu, c.diff);
                 if (lane == 0) {
                     if (prev_item >= 0) P.records[prev_item].X = dx;
                     if (live) {
@@ -518,21 +556,20 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                 }
             }
         }
-        parity ^= 1;
         prev_item = -1;
         x_carry = 0.f;
         if (!live) break;
         prev_item = item;
 
         // ---- second sweep over the parked e values ----
-        if (work && kSecondSweep) {
+        if (kSecondSweep) {
             const bool ok = tZa > 0.f && tZb > 0.f && tZa < 3.0e38f && tZb < 3.0e38f;   // false for NaN too
             const float iza = ok ? 1.0f / tZa : 0.f, izb = ok ? 1.0f / tZb : 0.f;
             const float ia = (ka == -INFINITY || !ok) ? 0.f : pow2_int(ka - Ka) * iza;
             const float ib = (kb == -INFINITY || !ok) ? 0.f : pow2_int(kb - Kb) * izb;
             uint64_t x2 = 0;
             float xt = 0.f;
-            // s = p + q + 2e-37 keeps lg2 finite where both terms vanish; the shift is below one ulp of any s that matters
+            // s = p + q + 1e-37 keeps lg2 finite where both terms vanish; the shift is below one ulp of any s that matters
             const uint64_t ia2 = pack2(ia, ia), ib2 = pack2(ib, ib), tiny2 = pack2(1e-37f, 1e-37f);
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
@@ -568,6 +605,12 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
             for (int m = 16; m > 0; m >>= 1) x += __shfl_xor_sync(0xffffffffu, x, m);
             x_carry = x;
         }
+
+        // ---- next pair ----
+        g += ns;
+        ++li;
+        item = next;
+        ra = ra_n; rb = rb_n; diff = diff_n;
     }
 
     // ---- release tensor memory ----
@@ -576,7 +619,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sh.tmem_base), "r"(kTmemCols) : "memory");
     }
-    cluster.sync();                                    // nobody leaves while a peer may still read its shared memory
+    cluster.sync();                                    // nobody leaves while a peer may still write to or read from it
 }
 
 // Occupancy twin: same block size, register bound and dynamic shared memory as the streaming
