@@ -61,10 +61,13 @@ int check_shape(int B, int G, int V) {
     return FSD_OK;
 }
 
-int finish_cluster_size(int V) {
-    // about 32 vocabulary entries per thread, at most the portable cluster size
+int finish_cluster_size(int B, int V) {
+    // about 32 vocabulary entries per thread, at most the portable cluster size, and no more CTAs
+    // than one wave of two per SM (148 SMs) when the batch is large
     int cs = 1;
-    while (cs < kMaxClusterSize && static_cast<long long>(cs) * kFinishThreads * 32 < V) cs <<= 1;
+    while (cs < kMaxClusterSize && static_cast<long long>(cs) * kFinishThreads * 32 < V &&
+           static_cast<long long>(B) * cs * 2 <= 2 * 148)
+        cs <<= 1;
     return cs;
 }
 
@@ -149,7 +152,7 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Pair
         fp.records = nullptr;
     }
 
-    const int cs = finish_cluster_size(fp.V);
+    const int cs = finish_cluster_size(fp.B, fp.V);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(fp.B) * cs, 1, 1);
     cfg.blockDim = dim3(kFinishThreads, 1, 1);

@@ -51,6 +51,8 @@ struct FinishExchange {        // what one CTA publishes to its cluster
 };
 struct FinishShared {
     FinishExchange slot;
+    double gather_d[kMaxClusterSize];   // one value per CTA of the cluster (see cluster_gather)
+    int gather_i[kMaxClusterSize];
     double exp_table[64];      // 2^(j/64)
     double red_d[32 * 2];
     float red_f[32 * 2];
@@ -93,6 +95,19 @@ __device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Fin
 #pragma unroll
     for (int r = 0; r < kMaxClusterSize; ++r) {
         if (r < cs) all[r] = cluster.map_shared_rank(&sh, r)->slot;
+    }
+    cluster.sync();
+}
+
+// Light exchange: every CTA publishes one double and one int; afterwards sh.gather_d / gather_i
+// hold the values of all CTAs, in rank order, in every CTA.  Two cluster barriers.
+__device__ __forceinline__ void cluster_gather(cg::cluster_group& cluster, FinishShared& sh, int cs, double v, int iv) {
+    if (threadIdx.x == 0) { sh.slot.d[0] = v; sh.slot.i[0] = iv; }
+    cluster.sync();
+    if (threadIdx.x < cs) {
+        const FinishShared* rs = cluster.map_shared_rank(&sh, threadIdx.x);
+        sh.gather_d[threadIdx.x] = rs->slot.d[0];
+        sh.gather_i[threadIdx.x] = rs->slot.i[0];
     }
     cluster.sync();
 }
@@ -257,6 +272,109 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const int k0 = k0l < V ? static_cast<int>(k0l) : V;
     const int k1 = (k0l + L) < V ? static_cast<int>(k0l + L) : V;
     FinishExchange mine, all[kMaxClusterSize];
+
+    // ---- fast path: inverse CDF over P_T (the FSD rule, and every bonus token) ----
+    if (!residual0 && !greedy) {
+        // Reference exponent k (log2 domain): the pair's record has it when this row was a pair's
+        // target row; otherwise one pass for the row maximum.
+        double kref = 0.0;
+        bool have_ref = false;
+        if (P.records != nullptr && !tree && n < G) {
+            const PairRecord* r = P.records + (static_cast<size_t>(b) * G + n);
+            const float rka = r->ka;
+            if ((r->state & kRecordStats) && isfinite(rka)) { kref = rka; have_ref = true; }
+        }
+        if (!have_ref) {
+            float m[1] = {-INFINITY};
+            for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int, float xa, float) { m[0] = fmaxf(m[0], xa); });
+            block_max<1>(m, sh.red_f);
+            cluster_gather(cluster, sh, cs, m[0], 0);
+            double M = -INFINITY;
+            for (int r = 0; r < cs; ++r) M = fmax(M, sh.gather_d[r]);
+            if (!isfinite(M)) {                           // no finite logit, or +inf: uniform over the cluster
+                if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.next_token[b] = -1; P.row_status[b] = status | FSD_ROW_NONFINITE; }
+                return;
+            }
+            kref = M * kLog2eD;
+        }
+        double csum = 0.0;
+        for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int, float xa, float) {
+            csum += exp2_table(fma(static_cast<double>(xa), kLog2eD, -kref), tab);
+        });
+        // inclusive / exclusive scan of the chunk sums over the CTA, fixed order
+        double incl = csum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        double excl = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) excl = 0.0;
+        if (lane == 31) sh.warp_tot[warp] = incl;
+        __syncthreads();
+        double wpre = 0.0, cta_tot = 0.0;
+        for (int w = 0; w < kFinishWarps; ++w) {
+            if (w == warp) wpre = cta_tot;
+            cta_tot += sh.warp_tot[w];
+        }
+        incl += wpre;
+        excl += wpre;
+        cluster_gather(cluster, sh, cs, cta_tot, 0);
+        double W = 0.0;
+        for (int r = 0; r < cs; ++r) W += sh.gather_d[r];
+        if (!(isfinite(W) && W > 0.0)) {                  // NaN logit (or nothing representable): uniform over the cluster
+            if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.next_token[b] = -1; P.row_status[b] = status | FSD_ROW_NONFINITE; }
+            return;
+        }
+        if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.row_status[b] = status; }
+        const double t = static_cast<double>(P.u_sample[b]) * W;
+        double cpre = 0.0, run = 0.0;
+        int owner = -1;
+        for (int r = 0; r < cs && owner < 0; ++r) {
+            cpre = run;
+            run += sh.gather_d[r];
+            if (run > t) owner = r;
+        }
+        auto last_with_weight = [&]() -> int {           // highest index of this thread's chunk whose weight is positive
+            int lastp = -1;
+            for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int k, float xa, float) {
+                if (exp2_table(fma(static_cast<double>(xa), kLog2eD, -kref), tab) > 0.0) lastp = k;
+            });
+            return lastp;
+        };
+        if (owner < 0) {                                  // t >= W after rounding (uniform): the last token that has weight
+            const int lp = __reduce_max_sync(0xffffffffu, last_with_weight());
+            if (lane == 0 && lp >= 0) atomicMax(&sh.last_pos, lp);
+            __syncthreads();
+            cluster_gather(cluster, sh, cs, 0.0, sh.last_pos);
+            int best = -1;
+            for (int r = 0; r < cs; ++r) best = sh.gather_i[r] > best ? sh.gather_i[r] : best;
+            if (rank == 0 && tid == 0) P.next_token[b] = best;
+            return;
+        }
+        if (owner != rank) return;
+        const double t_local = t - cpre;
+        if (csum > 0.0 && incl > t_local) atomicMin(&sh.cand, tid);
+        __syncthreads();
+        const int c = sh.cand;
+        if (c == 0x7fffffff) {                            // crossing lost to rounding inside this CTA
+            const int lp = __reduce_max_sync(0xffffffffu, last_with_weight());
+            if (lane == 0 && lp >= 0) atomicMax(&sh.last_pos, lp);
+            __syncthreads();
+            if (tid == 0) P.next_token[b] = sh.last_pos;
+        } else if (tid == c) {
+            double running = excl;
+            int tok = -1, lastp = -1;
+            for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int k, float xa, float) {
+                const double w = exp2_table(fma(static_cast<double>(xa), kLog2eD, -kref), tab);
+                running += w;
+                if (w > 0.0) lastp = k;
+                if (tok < 0 && running > t_local) tok = k;
+            });
+            P.next_token[b] = tok >= 0 ? tok : lastp;
+        }
+        return;
+    }
 
     // ---- CTA-local maxima (exact); for the greedy FSD choice also the argmax of the logits ----
     float mx[2] = {-INFINITY, -INFINITY};
