@@ -137,7 +137,7 @@ def run_reference(args, rank: int, world: int):
     """The reference arm: the CPU oracle on the host cores, each step a bounded sample of the workload."""
     if rank != 0:
         return
-    rows = 16
+    rows = args.ref_rows
     c = gi.make_config(WORKLOAD, B=rows)
     T = float(gi.CONFIGS[WORKLOAD].thresholds[0])
     for _ in range(max(args.warmup, 1)):
@@ -177,6 +177,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--copies", type=int, default=3)
+    ap.add_argument("--ref-rows", type=int, default=16, help="batch rows per step of the reference arm")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
