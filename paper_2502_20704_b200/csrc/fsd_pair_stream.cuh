@@ -185,6 +185,14 @@ __device__ __forceinline__ float pow2_int(float d) {
     return d < -126.f ? 0.f : __int_as_float((static_cast<int>(d) + 127) << 23);
 }
 
+// shared-memory counter increment that releases this thread's earlier writes and acquires the
+// other arrivers' (CTA scope); returns the old value
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+    int old;
+    asm volatile("atom.acq_rel.cta.shared::cta.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
+    return old;
+}
+
 // ---- cluster-scope mbarrier helpers (the statistics exchange) ------------------------------
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -433,8 +441,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
                     // this warp is done with the slot; the last warp to say so refills it
                     __syncwarp();
                     if (lane == 0) {
-                        __threadfence_block();
-                        if (atomicAdd(&sh.readers_done[slot], 1) == kStreamWarps - 1) {
+                        if (atom_add_acq_rel(&sh.readers_done[slot], 1) == kStreamWarps - 1) {
                             sh.readers_done[slot] = 0;
                             issue_stage(gs + kRing);
                         }
@@ -472,13 +479,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         int last = 0;
         if (lane == 0) {
             sh.ws[par][warp] = mine;
-            __threadfence_block();
-            last = atomicAdd(&sh.stats_done[par], 1) == kStreamWarps - 1;
+            last = atom_add_acq_rel(&sh.stats_done[par], 1) == kStreamWarps - 1;
             if (last) sh.stats_done[par] = 0;
         }
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
-            __threadfence_block();
             PartStats w;
             w.ka = -INFINITY; w.kb = -INFINITY; w.za = 0.f; w.zb = 0.f; w.sa = 0.f; w.sb = 0.f; w.kk = 0.f; w.x = 0.f; w.diff = 0;
             if (lane < kStreamWarps) w = sh.ws[par][lane];
