@@ -76,7 +76,7 @@ constexpr int kMaxDev = 64;
 
 template <int DT, int DIV>
 int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
-    static int max_clusters[kMaxDev][4] = {};       // per device, per log2(C); 0 = not yet queried
+    static int max_clusters[kMaxDev][5] = {};       // per device, per log2(C); 0 = not yet queried
     static std::mutex mu;
     auto kernel = fsd_pair_stream_kernel<DT, DIV>;
     int dev = 0;
@@ -105,6 +105,11 @@ int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
             if (cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
                 return FSD_ERR_CUDA;
+            if (C > 8) {                            // above the portable cluster size: opt in
+                if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+                    cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+                    return FSD_ERR_CUDA;
+            }
             cfg.gridDim = dim3(C, 1, 1);
             int n = 0;
             if (cudaOccupancyMaxActiveClusters(&n, fsd_stream_occupancy_twin, &cfg) != cudaSuccess || n < 1)
@@ -123,7 +128,7 @@ int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
 // on chip; 0 if the shape is not eligible (the generic kernel takes it).
 int stream_cluster_size(int nvec_row, bool vec) {
     if (!vec || nvec_row < 64) return 0;
-    for (int C = 1; C <= kMaxClusterSize; C <<= 1)
+    for (int C = 1; C <= kStreamMaxCluster; C <<= 1)
         if ((nvec_row + C - 1) / C <= kMaxVecPerCta) return C;
     return 0;
 }

@@ -113,13 +113,52 @@ __device__ __forceinline__ void cluster_gather(cg::cluster_group& cluster, Finis
 }
 
 // Divergence, accept bit and status of one pair from the streaming kernel's totals.
+// A pair's totals from the parts its record holds (one per CTA of the streaming cluster), in
+// double: Z = sum 2^y, S = sum 2^y * y, K = sum 2^ya (ya - yb), all relative to the largest
+// part reference (the parts' references are integers, so the factors are exact powers of two).
+struct PairTotals {
+    double Za, Zb, Sa, Sb, K, X;
+    float ka, kb;
+    uint32_t differ;
+};
+__device__ inline PairTotals fold_record(const PairRecord& rec, int div) {
+    PairTotals t;
+    t.Za = 0.0; t.Zb = 0.0; t.Sa = 0.0; t.Sb = 0.0; t.K = 0.0; t.X = 0.0; t.differ = 0;
+    const int n = static_cast<int>(rec.ncta) < kStreamMaxCluster ? static_cast<int>(rec.ncta) : kStreamMaxCluster;
+    float ka = -INFINITY, kb = -INFINITY;
+    for (int r = 0; r < n; ++r) {                       // NaN references win
+        const float a = rec.part[r].ka, b = rec.part[r].kb;
+        ka = (a != a || ka != ka) ? __int_as_float(0x7fc00000) : fmaxf(ka, a);
+        kb = (b != b || kb != kb) ? __int_as_float(0x7fc00000) : fmaxf(kb, b);
+    }
+    t.ka = ka; t.kb = kb;
+    for (int r = 0; r < n; ++r) {
+        const Stats c = rec.part[r];
+        const double da = c.ka == -INFINITY ? 0.0 : static_cast<double>(c.ka) - ka;
+        const double db = c.kb == -INFINITY ? 0.0 : static_cast<double>(c.kb) - kb;
+        const double fa = c.ka == -INFINITY ? 0.0 : (da < -2000.0 ? 0.0 : scalbn(1.0, static_cast<int>(da)));
+        const double fb = c.kb == -INFINITY ? 0.0 : (db < -2000.0 ? 0.0 : scalbn(1.0, static_cast<int>(db)));
+        t.Za += fa * c.za; t.Zb += fb * c.zb;
+        if (div == FSD_DIV_KL) {
+            t.K += c.s0 == INFINITY ? static_cast<double>(INFINITY) : fa * (static_cast<double>(c.s0) + (da - db) * c.za);
+        } else {
+            t.Sa += fa * (static_cast<double>(c.s0) + da * c.za);
+            t.Sb += fb * (static_cast<double>(c.sb) + db * c.zb);
+        }
+        t.X += rec.x[r];
+        t.differ |= c.diff;
+    }
+    return t;
+}
+
 __device__ inline void judge_record(const FinishParams& P, int item, const void* a_row, const void* b_row, int dt,
                                     float& D_out, int& bit_out, int& st_out) {
-    const PairRecord r = P.records[item];
-    if (r.state & kRecordBadTree) {
+    const PairRecord& rec = P.records[item];
+    if (rec.state & kRecordBadTree) {
         D_out = __int_as_float(0x7fc00000); bit_out = 0; st_out = FSD_ROW_BADTREE;
         return;
     }
+    const PairTotals r = fold_record(rec, P.div);
     const bool finite = isfinite(r.ka) && isfinite(r.kb) && r.Za > 0.0 && r.Zb > 0.0 && isfinite(r.Za) && isfinite(r.Zb);
     float D = __int_as_float(0x7fc00000);
     if (finite) D = r.differ ? static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X)) : 0.0f;
@@ -281,8 +320,16 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         bool have_ref = false;
         if (P.records != nullptr && !tree && n < G) {
             const PairRecord* r = P.records + (static_cast<size_t>(b) * G + n);
-            const float rka = r->ka;
-            if ((r->state & kRecordStats) && isfinite(rka)) { kref = rka; have_ref = true; }
+            if (r->state & kRecordStats) {                // any common reference near the maximum serves
+                float rka = -INFINITY;
+                bool nan = false;
+                for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
+                    const float a = r->part[c].ka;
+                    nan = nan || a != a;
+                    rka = fmaxf(rka, a);
+                }
+                if (!nan && isfinite(rka)) { kref = rka; have_ref = true; }
+            }
         }
         if (!have_ref) {
             float m[1] = {-INFINITY};

@@ -4,51 +4,74 @@
 // (C = 1, 2, 4 or 8, the smallest that lets a CTA's slice fit on chip).  Clusters are
 // persistent and walk the pair list round-robin.  Per pair, each CTA
 //   1. receives its slice of both rows in shared memory through a ring of bulk asynchronous
-//      copies (cp.async.bulk + mbarrier; the next pair's slices stream in meanwhile),
-//   2. sweeps the slice once from shared memory for each thread's exact maximum and a
-//      bitwise "rows differ" flag,
-//   3. sweeps it again computing e = 2^(logit * log2e - k) with one MUFU ex2 per logit, where k
-//      is the thread's maximum rounded up to an integer in the log2 domain (so every later
-//      change of reference is an exact power of two), the sums Z = sum e and S = sum e*y (and
-//      the KL sum), and parks the e values in tensor memory (64 per thread) and registers (16),
-//   4. combines (k, Z, S) over threads and warps, then -- one CTA barrier and one cluster
-//      barrier later -- over the CTA and, through distributed shared memory, the cluster,
-//   5. sweeps the parked e values: p = e_a/Z_a, q = e_b/Z_b; JS needs sum (p+q) log2(p+q) (one
+//      copies (cp.async.bulk + mbarrier).  A ring slot is refilled as soon as its last reader
+//      is done, so the next pair's slices stream in while this pair is finished;
+//   2. sweeps each stage once as it lands: e = 2^(logit * log2e - k) with one MUFU ex2 per
+//      logit, the sums Z = sum e and S = sum e*y (or the KL sum), a bitwise "rows differ" flag,
+//      and parks the e values in tensor memory (128 per thread) and registers (32).  k is a
+//      per-thread integer reference in the log2 domain, taken from the thread's first finite
+//      logits and moved -- with an exact power-of-two rescale of what has been summed and parked
+//      -- only if a later logit exceeds it by more than 2^30, so no separate maximum pass over
+//      the slice is needed and every change of reference is exact;
+//   3. combines (k, Z, S) over threads and warps; one combiner warp per CTA (rotating) folds
+//      the warps' statistics, sends them to every CTA of the cluster with asynchronous
+//      distributed-shared-memory stores that signal the receiver's mbarrier, folds what the
+//      cluster sent and wakes the CTA (named barriers: waiting warps issue nothing);
+//   4. sweeps the parked e values: p = e_a/Z_a, q = e_b/Z_b; JS needs sum (p+q) log2(p+q) (one
 //      MUFU lg2 per pair), TV needs sum |p - q|; KL needs no second sweep.
-// The cluster's rank-0 CTA writes the pair's totals to a 64-byte record; the finish kernel
-// turns records into divergences and accept bits, so no double-precision transcendental runs
-// here.  The logits are never touched again after step 3: HBM traffic is the algorithmic
-// minimum.  The special-function pipe (1 ex2 per logit + 1 lg2 per pair) is the co-bottleneck,
-// which is why e values are kept rather than recomputed.  Two CTAs share an SM so that one
-// CTA's barrier bubbles are filled by the other.
+// The cluster's rank-0 CTA leaves the CTAs' statistics in the pair's record; the finish kernel
+// folds them in double precision and turns them into divergences and accept bits, so no
+// double-precision arithmetic runs here.  HBM traffic is the algorithmic minimum.  The
+// special-function pipe (1 ex2 per logit + 1 lg2 per pair) and instruction issue are the
+// co-bottlenecks, which is why e values are kept rather than recomputed, and why a thread
+// owns two vectors per row and stage (independent work to overlap its own latencies) with two
+// CTAs of 256 threads and 128 registers per SM.
 #pragma once
 
 #include "fsd_device.cuh"
 
 namespace fsd {
 
-constexpr int kStreamThreads = 512;
+constexpr int kStreamThreads = 256;
 constexpr int kStreamWarps = kStreamThreads / 32;
 constexpr int kRing = 6;                                   // stages in the shared-memory ring
-constexpr int kStageRowBytes = kStreamThreads * 16;        // one 16-byte vector per thread and row
+constexpr int kVecPerThread = 2;                           // 16-byte vectors per thread, row and stage
+constexpr int kStageVecs = kStreamThreads * kVecPerThread; // vectors per row and stage
+constexpr int kStageRowBytes = kStageVecs * 16;
 constexpr int kStageBytes = 2 * kStageRowBytes;
 constexpr int kMaxStagesPerPair = kRing - 1;               // a pair's slice must be resident at once
-constexpr int kTmemCols = 256;                             // per CTA: 16 warps -> 4 per lane quarter x 64 columns
-constexpr int kTmemPerThread = 64;
-constexpr int kMaxVecPerCta = kMaxStagesPerPair * kStreamThreads;
-constexpr int kMaxClusterSize = 8;
+constexpr int kTmemCols = 256;                             // per CTA: 8 warps -> 2 per lane quarter x 128 columns
+constexpr int kTmemPerThread = 128;
+constexpr int kMaxVecPerCta = kMaxStagesPerPair * kStageVecs;
+constexpr int kMaxClusterSize = 8;                        // finish kernel (portable size)
+constexpr int kStreamMaxCluster = 8;                       // streaming kernel
+constexpr int kStreamCtasPerSm = 2;
 constexpr uint32_t kSpinLimit = 1u << 24;                  // polls before a wait gives up
 
-// Totals of one pair, written by the streaming kernel and read by the finish kernel.
-//   Z = sum 2^y, S = sum 2^y * y, K = sum 2^ya (ya - yb), with y = logit*log2e - k and k the
-//   integer reference of the row; X = second-sweep sum (JS: sum s log2 s, TV: sum |p - q|).
-struct PairRecord {
-    double Za, Zb, Sa, Sb, K, X;
-    float ka, kb;              // integer-valued references (log2 domain); -inf: no finite logit; NaN: row holds a NaN
-    uint32_t differ;           // 0: the two rows are bitwise identical
-    uint32_t state;            // kRecordStats | kRecordBadTree
+// Partial statistics of one (target row, draft row) pair: of a warp, of a CTA, or -- in a
+// pair's record -- of each CTA of the cluster that streamed the pair.
+//   z = sum 2^y, s = sum 2^y * y with y = logit*log2e - k and k the integer reference (log2
+//   domain) the sums are relative to.  s0 is the target row's s for JS and the KL sum
+//   sum 2^ya (ya - yb) for KL.
+struct alignas(16) Stats {
+    float ka, kb;              // references; -inf: no finite logit seen; NaN: a NaN logit
+    float za, zb;
+    float s0, sb;
+    float x;                   // second-sweep sum of the PREVIOUS pair (in flight only)
+    uint32_t diff;             // 0: the two rows are bitwise identical so far
 };
-static_assert(sizeof(PairRecord) == 64, "PairRecord is one 64-byte line");
+static_assert(sizeof(Stats) == 32, "Stats travels as two 16-byte stores");
+
+// What the streaming kernel leaves per pair for the finish kernel, which folds the parts in
+// double precision (second-sweep sums: JS sum s log2 s, TV sum |p - q|).
+struct alignas(16) PairRecord {
+    Stats part[kStreamMaxCluster];
+    float x[kStreamMaxCluster];  // each CTA's second-sweep sum of this pair
+    uint32_t ncta;             // parts in use
+    uint32_t state;            // kRecordStats | kRecordBadTree
+    uint32_t pad[2];
+};
+static_assert(sizeof(PairRecord) == 304, "PairRecord layout");
 constexpr uint32_t kRecordStats = 1, kRecordBadTree = 2;
 
 struct StreamParams {
@@ -185,15 +208,76 @@ __device__ __forceinline__ float pow2_int(float d) {
     return d < -126.f ? 0.f : __int_as_float((static_cast<int>(d) + 127) << 23);
 }
 
-// shared-memory counter increment that releases this thread's earlier writes and acquires the
-// other arrivers' (CTA scope); returns the old value
-__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+// ---- in-stream references ---------------------------------------------------------------------
+// A thread keeps, per row, the largest logit its reference may meet without moving: bf16 rows
+// hold it as a packed pair so that one packed maximum tests a whole vector.  -1e30 is what -inf
+// logits are read as, so "nothing finite seen yet" is a limit of exactly that.
+template <int DT> __device__ __forceinline__ uint32_t unset_limit() {
+    return DT == FSD_BF16 ? 0xF149F149u : __float_as_uint(-1.0e30f);
+}
+// limit for a reference taken from maximum m: m + 30 ln 2, rounded to the row's type (rounding
+// can add at most another 30 ln 2 before it snaps back to m itself, so 2^y stays below 2^61)
+template <int DT> __device__ __forceinline__ uint32_t reference_limit(float m) {
+    const float lim = m + 20.7944f;
+    if constexpr (DT == FSD_BF16) {
+        uint32_t r;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(lim), "f"(lim));
+        return r;
+    } else {
+        return __float_as_uint(lim);
+    }
+}
+// Multiplies the e values a warp has parked in tensor memory for stages 0..n-1 by fa (first
+// half of each stage: target row) and fb (second half: draft row).  Warp-collective.
+template <int EPT>
+__device__ __noinline__ void rescale_parked(uint32_t taddr, int n, float fa, float fb) {
+    tmem_wait_st();
+    for (int t = 0; t < n; ++t) {
+        float e[EPT];
+        tmem_ld<EPT>(taddr + t * EPT, e);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < EPT / 2; ++j) { e[j] *= fa; e[EPT / 2 + j] *= fb; }
+        tmem_st<EPT>(taddr + t * EPT, e);
+    }
+    tmem_wait_st();
+}
+
+// A KL partial sum brought to another reference: +inf (a logit with p > 0 = q) stays +inf even
+// when the factor underflows to 0
+__device__ __forceinline__ float scale_kl(float f, float v) { return v == INFINITY ? v : f * v; }
+
+// 16-byte store into CTA `rank`'s copy of `dst` that, on landing, counts 16 bytes on that CTA's
+// copy of barrier `bar`: the store carries its own signal, the sender neither fences nor waits
+__device__ __forceinline__ void st_async_remote(void* dst, uint64_t* bar, uint32_t rank, float a, float b, float c, float d) {
+    uint32_t rdst, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rdst) : "r"(smem_u32(dst)), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(bar)), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(rdst), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)), "r"(__float_as_uint(d)), "r"(rbar)
+                 : "memory");
+}
+// CTA-wide named barriers: waiting warps issue nothing.  `arrive` counts the warp in without
+// waiting; `sync` waits until kStreamThreads threads have arrived or synced.
+__device__ __forceinline__ void named_arrive(int id) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "n"(kStreamThreads) : "memory");
+}
+__device__ __forceinline__ void named_sync(int id) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(kStreamThreads) : "memory");
+}
+constexpr int kBarPosted = 1, kBarTotals = 2;
+
+// Shared-memory counter increment, returns the old value.  Relaxed: a warp's reads of a ring
+// slot have completed by the time it counts itself out (their values were consumed), and the
+// thread that refills the slot orders its own reset of the counter before the copy through the
+// proxy fence and the barrier it arms.
+__device__ __forceinline__ int atom_add_relaxed(int* p, int v) {
     int old;
-    asm volatile("atom.acq_rel.cta.shared::cta.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
+    asm volatile("atom.relaxed.cta.shared::cta.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
     return old;
 }
 
-// ---- cluster-scope mbarrier helpers (the statistics exchange) ------------------------------
+// ---- cluster-scope mbarrier wait (the statistics exchange) ------------------------------------
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -212,36 +296,26 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
     dead = true;
     return false;
 }
-// arrive (release, cluster scope) on the same-named barrier of CTA `rank` of this cluster
-__device__ __forceinline__ void mbar_arrive_remote(uint64_t* bar, uint32_t rank) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
-}
 
 // ---- shared-memory layout ---------------------------------------------------------------
-struct PartStats {             // statistics of a warp (in ws) or of a CTA (in xch)
-    float ka, kb;              // references
-    float za, zb, sa, sb, kk;  // sums relative to the references
-    float x;                   // second-sweep sum of the PREVIOUS pair
-    uint32_t diff;
-};
 struct StreamShared {
     uint64_t full[kRing];      // a ring stage has landed
-    uint64_t xbar[2];          // every CTA of the cluster has delivered its statistics (per parity)
+    uint64_t xbar[2];          // all CTAs' statistics have landed here (per parity): 1 arrival + C * 32 bytes
     int readers_done[kRing];   // warps that have finished reading the slot's current stage
-    int stats_done[2];         // warps that have posted their statistics (per parity)
     uint32_t tmem_base;
-    PartStats ws[2][kStreamWarps];
-    PartStats xch[2][kMaxClusterSize];     // written by the peers (and by this CTA for its own rank)
+    alignas(16) float tot[4];  // cluster totals of the current pair: Ka, Kb, Za, Zb
+    Stats ws[kStreamWarps];    // the warps' statistics of the current pair
+    Stats xch[2][kStreamMaxCluster];         // written by the peers (and by this CTA for its own rank)
 };
 constexpr size_t kStreamSmemBytes = kRing * kStageBytes + sizeof(StreamShared) + 128;
 
 template <int DT, int DIV>
-__global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(StreamParams P) {
+__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_stream_kernel(StreamParams P) {
     constexpr int EPV = Logit<DT>::kPerVec;          // logits per 16-byte vector
-    constexpr int EPT = 2 * EPV;                     // e values per thread and stage (both rows)
-    constexpr int NT = (kTmemPerThread / EPT) < kMaxStagesPerPair ? (kTmemPerThread / EPT) : kMaxStagesPerPair;
+    constexpr int EPT = 2 * EPV;                     // e values per thread and vector position (both rows)
+    constexpr int VPT = kVecPerThread;
+    constexpr int EPS = VPT * EPT;                   // e values per thread and stage
+    constexpr int NT = (kTmemPerThread / EPS) < kMaxStagesPerPair ? (kTmemPerThread / EPS) : kMaxStagesPerPair;
     constexpr int NR = kMaxStagesPerPair - NT;       // stages kept in registers
     constexpr bool kSecondSweep = DIV != FSD_DIV_KL;
     constexpr float kClamp = -1.0e30f;               // -inf logits are read as this: 2^y = 0 and 0 * y = 0 stay finite
@@ -260,15 +334,14 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     const int base = P.nvec_row / C, rem = P.nvec_row % C;
     const int vbeg = rank * base + (rank < rem ? rank : rem);
     const int vcnt = base + (rank < rem ? 1 : 0);
-    const int ns = (vcnt + kStreamThreads - 1) / kStreamThreads;     // stages per pair (<= kMaxStagesPerPair)
+    const int ns = (vcnt + kStageVecs - 1) / kStageVecs;             // stages per pair (<= kMaxStagesPerPair)
     const size_t row_bytes = static_cast<size_t>(P.nvec_row) * 16;
 
     // ---- set-up: barriers, tensor memory ----
     if (blockIdx.x == 0 && tid == 0) *P.timeout_flag = 0;   // a wait needs far longer to run out than this store takes
     if (tid == 0) {
         for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); sh.readers_done[s] = 0; }
-        mbar_init(&sh.xbar[0], C); mbar_init(&sh.xbar[1], C);
-        sh.stats_done[0] = 0; sh.stats_done[1] = 0;
+        mbar_init(&sh.xbar[0], 1); mbar_init(&sh.xbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -279,8 +352,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     cluster.sync();                                  // barriers of every CTA exist before any peer arrives on them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // warp w owns tensor-memory lanes 32*(w%4)..+31 and columns 64*(w/4)..+63
-    const uint32_t taddr = sh.tmem_base + (static_cast<uint32_t>(32 * (warp & 3)) << 16) + static_cast<uint32_t>(64 * (warp >> 2));
+    // warp w owns tensor-memory lanes 32*(w%4)..+31 and columns kTmemPerThread*(w/4)..
+    const uint32_t taddr = sh.tmem_base + (static_cast<uint32_t>(32 * (warp & 3)) << 16) + static_cast<uint32_t>(kTmemPerThread * (warp >> 2));
 
     bool dead = false;                               // a bounded wait of this thread ran out
 
@@ -301,8 +374,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         const char* a_row = static_cast<const char*>(P.target) + (static_cast<size_t>(b) * (P.G + 1) + trow) * row_bytes;
         const char* b_row = static_cast<const char*>(P.draft) + (static_cast<size_t>(b) * P.G + i) * row_bytes;
         const uint32_t slot = gg % kRing;
-        const int v0 = static_cast<int>(s) * kStreamThreads;
-        const int nv = (vcnt - v0) < kStreamThreads ? (vcnt - v0) : kStreamThreads;
+        const int v0 = static_cast<int>(s) * kStageVecs;
+        const int nv = (vcnt - v0) < kStageVecs ? (vcnt - v0) : kStageVecs;
         const uint32_t bytes = static_cast<uint32_t>(nv) * 16;
         unsigned char* dst = ring + slot * kStageBytes;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of the slot precede the async writes
@@ -315,44 +388,12 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
     }
     __syncwarp();
 
-    // ---- sweep A: exact thread maxima and the bitwise difference flag of the pair starting at stage gA ----
-    auto sweep_a = [&](uint32_t gA, float& ra, float& rb, uint32_t& diff) {
-        ra = -INFINITY; rb = -INFINITY; diff = 0;
-#pragma unroll
-        for (int s = 0; s < kMaxStagesPerPair; ++s) {
-            if (s < ns) {
-                const uint32_t gs = gA + s, slot = gs % kRing;
-                mbar_wait(&sh.full[slot], (gs / kRing) & 1, P.timeout_flag, dead);
-                if (s * kStreamThreads + tid < vcnt) {
-                    const unsigned char* st = ring + slot * kStageBytes + tid * 16;
-                    const uint4 va = *reinterpret_cast<const uint4*>(st);
-                    const uint4 vb = *reinterpret_cast<const uint4*>(st + kStageRowBytes);
-                    diff |= (va.x ^ vb.x) | (va.y ^ vb.y) | (va.z ^ vb.z) | (va.w ^ vb.w);
-                    if constexpr (DT == FSD_BF16) {
-                        const uint32_t ma = bf16x2_max_nan(bf16x2_max_nan(va.x, va.y), bf16x2_max_nan(va.z, va.w));
-                        const uint32_t mb = bf16x2_max_nan(bf16x2_max_nan(vb.x, vb.y), bf16x2_max_nan(vb.z, vb.w));
-                        ra = fmax_nan(ra, fmax_nan(bf16_lo(ma), bf16_hi(ma)));
-                        rb = fmax_nan(rb, fmax_nan(bf16_lo(mb), bf16_hi(mb)));
-                    } else {
-                        ra = fmax_nan(ra, fmax_nan(fmax_nan(__uint_as_float(va.x), __uint_as_float(va.y)),
-                                                   fmax_nan(__uint_as_float(va.z), __uint_as_float(va.w))));
-                        rb = fmax_nan(rb, fmax_nan(fmax_nan(__uint_as_float(vb.x), __uint_as_float(vb.y)),
-                                                   fmax_nan(__uint_as_float(vb.z), __uint_as_float(vb.w))));
-                    }
-                }
-            }
-        }
-    };
-
-    float ereg[(NR > 0 ? NR : 1) * EPT];
+    float ereg[(NR > 0 ? NR : 1) * EPS];
     uint32_t g = 0;                                  // first ring stage of the current pair
     uint32_t li = 0;                                 // pairs this cluster has finished
     float x_carry = 0.f;                             // previous pair's second-sweep sum of this warp
     int prev_item = -1;                              // pair whose second-sweep sum is still to be published
     int item = cluster_id;
-    float ra = -INFINITY, rb = -INFINITY;
-    uint32_t diff = 0;
-    if (item < P.n_items) sweep_a(0, ra, rb, diff);
 
     for (;;) {
         const bool live = item < P.n_items;          // one extra round publishes the last pair's second sweep
@@ -368,199 +409,250 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
 
         // ---- sweep B: exponentials, sums, park the e values; then this warp's statistics ----
         float ka = -INFINITY, kb = -INFINITY;
-        PartStats mine;
-        mine.ka = -INFINITY; mine.kb = -INFINITY; mine.za = 0.f; mine.zb = 0.f; mine.sa = 0.f; mine.sb = 0.f; mine.kk = 0.f;
+        Stats mine;
+        mine.ka = -INFINITY; mine.kb = -INFINITY; mine.za = 0.f; mine.zb = 0.f; mine.s0 = 0.f; mine.sb = 0.f;
         mine.diff = 0;
         if (live) {
             float kk = 0.f;
+            uint32_t diff = 0;
             uint64_t za2 = 0, zb2 = 0, sa2 = 0, sb2 = 0;     // packed (even, odd) partial sums
-            // integer references in the log2 domain: y = logit*log2e - k <= 0 up to rounding
-            ka = ra == -INFINITY ? -INFINITY : ceilf(ra * kLog2e);
-            kb = rb == -INFINITY ? -INFINITY : ceilf(rb * kLog2e);
-            const float ca = ra == -INFINITY ? 0.f : -ka, cb = rb == -INFINITY ? 0.f : -kb;
-            const uint64_t l2 = pack2(kLog2e, kLog2e), ca2 = pack2(ca, ca), cb2 = pack2(cb, cb);
+            // Integer references in the log2 domain, y = logit*log2e - k.  A thread takes k from the
+            // first vector that holds a finite logit and keeps it while no later logit exceeds it by
+            // more than about 2^30 (2^60 at most); a larger one moves the reference and rescales what
+            // has been summed and parked, by an exact power of two.
+            uint32_t lima = unset_limit<DT>(), limb = unset_limit<DT>(); // a vector maximum above this moves the reference
+            uint64_t ca2 = 0, cb2 = 0;                       // packed -k (0 while no finite logit has been seen)
+            const uint64_t l2 = pack2(kLog2e, kLog2e);
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
                 if (s < ns) {
                     const uint32_t gs = g + s, slot = gs % kRing;
-                    float e[EPT];
-                    if (s * kStreamThreads + tid < vcnt) {
-                        const unsigned char* st = ring + slot * kStageBytes + tid * 16;
-                        uint4 va = *reinterpret_cast<const uint4*>(st);
-                        uint4 vb = *reinterpret_cast<const uint4*>(st + kStageRowBytes);
-                        float xa[EPV], xb[EPV];
+                    mbar_wait(&sh.full[slot], (gs / kRing) & 1, P.timeout_flag, dead);
+                    // this thread's vectors of the stage: v * kStreamThreads + tid, v < VPT
+                    uint4 va[VPT], vb[VPT];
+                    bool has[VPT];
+                    float ma = 0.f, mb = 0.f;                // maxima of this thread's vectors of the stage
+                    bool fire_a = false, fire_b = false;
+                    {
+                        uint32_t pa = unset_limit<DT>(), pb = unset_limit<DT>();   // -1e30: below every clamped logit
+#pragma unroll
+                        for (int v = 0; v < VPT; ++v) {
+                            has[v] = s * kStageVecs + v * kStreamThreads + tid < vcnt;
+                            va[v] = make_uint4(0, 0, 0, 0); vb[v] = make_uint4(0, 0, 0, 0);
+                            if (has[v]) {
+                                const unsigned char* st = ring + slot * kStageBytes + (v * kStreamThreads + tid) * 16;
+                                va[v] = *reinterpret_cast<const uint4*>(st);
+                                vb[v] = *reinterpret_cast<const uint4*>(st + kStageRowBytes);
+                                diff |= (va[v].x ^ vb[v].x) | (va[v].y ^ vb[v].y) | (va[v].z ^ vb[v].z) | (va[v].w ^ vb[v].w);
+                                if constexpr (DT == FSD_BF16) {
+                                    constexpr uint32_t kClamp2 = 0xF149F149u;     // bf16x2 (-1e30, -1e30); NaN passes through
+                                    va[v].x = bf16x2_max_nan(va[v].x, kClamp2); va[v].y = bf16x2_max_nan(va[v].y, kClamp2);
+                                    va[v].z = bf16x2_max_nan(va[v].z, kClamp2); va[v].w = bf16x2_max_nan(va[v].w, kClamp2);
+                                    if constexpr (DIV != FSD_DIV_KL) {            // KL needs the draft's -inf: q = 0 < p gives +inf
+                                        vb[v].x = bf16x2_max_nan(vb[v].x, kClamp2); vb[v].y = bf16x2_max_nan(vb[v].y, kClamp2);
+                                        vb[v].z = bf16x2_max_nan(vb[v].z, kClamp2); vb[v].w = bf16x2_max_nan(vb[v].w, kClamp2);
+                                    }
+                                    pa = bf16x2_max_nan(pa, bf16x2_max_nan(bf16x2_max_nan(va[v].x, va[v].y), bf16x2_max_nan(va[v].z, va[v].w)));
+                                    pb = bf16x2_max_nan(pb, bf16x2_max_nan(bf16x2_max_nan(vb[v].x, vb[v].y), bf16x2_max_nan(vb[v].z, vb[v].w)));
+                                } else {
+                                    const float m1 = fmax_nan(fmax_nan(__uint_as_float(va[v].x), __uint_as_float(va[v].y)),
+                                                              fmax_nan(__uint_as_float(va[v].z), __uint_as_float(va[v].w)));
+                                    const float m2 = fmax_nan(fmax_nan(__uint_as_float(vb[v].x), __uint_as_float(vb[v].y)),
+                                                              fmax_nan(__uint_as_float(vb[v].z), __uint_as_float(vb[v].w)));
+                                    pa = __float_as_uint(fmax_nan(__uint_as_float(pa), m1));
+                                    pb = __float_as_uint(fmax_nan(__uint_as_float(pb), m2));
+                                }
+                            }
+                        }
                         if constexpr (DT == FSD_BF16) {
-                            constexpr uint32_t kClamp2 = 0xF149F149u;     // bf16x2 (-1e30, -1e30)
-                            va.x = bf16x2_max(va.x, kClamp2); va.y = bf16x2_max(va.y, kClamp2);
-                            va.z = bf16x2_max(va.z, kClamp2); va.w = bf16x2_max(va.w, kClamp2);
-                            if constexpr (DIV != FSD_DIV_KL) {            // KL needs the draft's -inf: q = 0 < p gives +inf
-                                vb.x = bf16x2_max(vb.x, kClamp2); vb.y = bf16x2_max(vb.y, kClamp2);
-                                vb.z = bf16x2_max(vb.z, kClamp2); vb.w = bf16x2_max(vb.w, kClamp2);
-                            }
+                            fire_a = bf16x2_max_nan(pa, lima) != lima;
+                            fire_b = bf16x2_max_nan(pb, limb) != limb;
+                            if (fire_a) ma = fmax_nan(bf16_lo(pa), bf16_hi(pa));
+                            if (fire_b) mb = fmax_nan(bf16_lo(pb), bf16_hi(pb));
+                        } else {
+                            ma = __uint_as_float(pa); mb = __uint_as_float(pb);
+                            fire_a = !(ma <= __uint_as_float(lima));      // NaN moves the reference too
+                            fire_b = !(mb <= __uint_as_float(limb));
                         }
-                        unpack_vec<DT>(va, xa);
-                        unpack_vec<DT>(vb, xb);
-#pragma unroll
-                        for (int j = 0; j < EPV; j += 2) {
-                            float a0 = xa[j], a1 = xa[j + 1], b0 = xb[j], b1 = xb[j + 1];
-                            if constexpr (DT == FSD_F32) {
-                                a0 = fmaxf(a0, kClamp); a1 = fmaxf(a1, kClamp);
-                                if constexpr (DIV != FSD_DIV_KL) { b0 = fmaxf(b0, kClamp); b1 = fmaxf(b1, kClamp); }
-                            }
-                            const uint64_t ya2 = fma2(pack2(a0, a1), l2, ca2), yb2 = fma2(pack2(b0, b1), l2, cb2);
-                            float ya0, ya1, yb0, yb1;
-                            unpack2(ya2, ya0, ya1);
-                            unpack2(yb2, yb0, yb1);
-                            const float ea0 = ex2(ya0), ea1 = ex2(ya1), eb0 = ex2(yb0), eb1 = ex2(yb1);
-                            const uint64_t ea2 = pack2(ea0, ea1), eb2 = pack2(eb0, eb1);
-                            za2 = add2(za2, ea2);
-                            zb2 = add2(zb2, eb2);
-                            if constexpr (DIV == FSD_DIV_JS) {
-                                sa2 = fma2(ea2, ya2, sa2);
-                                sb2 = fma2(eb2, yb2, sb2);
-                            }
-                            if constexpr (DIV == FSD_DIV_KL) {
-                                if (ea0 > 0.f) kk = fmaf(ea0, ya0 - yb0, kk);
-                                if (ea1 > 0.f) kk = fmaf(ea1, ya1 - yb1, kk);
-                            }
-                            e[j] = ea0; e[j + 1] = ea1;
-                            e[EPV + j] = eb0; e[EPV + j + 1] = eb1;
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < EPT; ++j) e[j] = 0.f;
                     }
-                    if constexpr (kSecondSweep) {
-                        if (s < NT) {
-                            tmem_st<EPT>(taddr + s * EPT, e);
+                    __syncwarp();
+                    if (__any_sync(0xffffffffu, fire_a || fire_b)) {
+                        // rare after a pair's first vector: lanes that did not fire scale by 1
+                        const float nka = fire_a ? ceilf(ma * kLog2e) : ka, nkb = fire_b ? ceilf(mb * kLog2e) : kb;
+                        const float da = ka == -INFINITY ? 0.f : ka - nka, db = kb == -INFINITY ? 0.f : kb - nkb;
+                        const float fa = ka == -INFINITY ? 0.f : pow2_int(da), fb = kb == -INFINITY ? 0.f : pow2_int(db);
+                        const uint64_t fa2 = pack2(fa, fa), fb2 = pack2(fb, fb);
+                        if constexpr (DIV == FSD_DIV_KL) kk = scale_kl(fa, fmaf(da - db, sum2(za2), kk));
+                        sa2 = mul2(fma2(za2, pack2(da, da), sa2), fa2); za2 = mul2(za2, fa2);
+                        sb2 = mul2(fma2(zb2, pack2(db, db), sb2), fb2); zb2 = mul2(zb2, fb2);
+                        if constexpr (kSecondSweep) {
+                            if (s > 0) rescale_parked<EPT>(taddr, (s < NT ? s : NT) * VPT, fa, fb);
+#pragma unroll
+                            for (int t = NT; t < s; ++t) {
+#pragma unroll
+                                for (int v = 0; v < VPT; ++v) {
+#pragma unroll
+                                    for (int j = 0; j < EPV; ++j) {
+                                        ereg[(t - NT) * EPS + v * EPT + j] *= fa;
+                                        ereg[(t - NT) * EPS + v * EPT + EPV + j] *= fb;
+                                    }
+                                }
+                            }
+                        }
+                        if (fire_a) lima = reference_limit<DT>(ma);
+                        if (fire_b) limb = reference_limit<DT>(mb);
+                        ka = nka; kb = nkb;
+                        const float ca = ka == -INFINITY ? 0.f : -ka, cb = kb == -INFINITY ? 0.f : -kb;
+                        ca2 = pack2(ca, ca); cb2 = pack2(cb, cb);
+                    }
+                    float e[VPT][EPT];
+#pragma unroll
+                    for (int v = 0; v < VPT; ++v) {
+                        if (has[v]) {
+                            float xa[EPV], xb[EPV];
+                            unpack_vec<DT>(va[v], xa);
+                            unpack_vec<DT>(vb[v], xb);
+#pragma unroll
+                            for (int j = 0; j < EPV; j += 2) {
+                                float a0 = xa[j], a1 = xa[j + 1], b0 = xb[j], b1 = xb[j + 1];
+                                if constexpr (DT == FSD_F32) {
+                                    a0 = fmaxf(a0, kClamp); a1 = fmaxf(a1, kClamp);
+                                    if constexpr (DIV != FSD_DIV_KL) { b0 = fmaxf(b0, kClamp); b1 = fmaxf(b1, kClamp); }
+                                }
+                                const uint64_t ya2 = fma2(pack2(a0, a1), l2, ca2), yb2 = fma2(pack2(b0, b1), l2, cb2);
+                                float ya0, ya1, yb0, yb1;
+                                unpack2(ya2, ya0, ya1);
+                                unpack2(yb2, yb0, yb1);
+                                const float ea0 = ex2(ya0), ea1 = ex2(ya1), eb0 = ex2(yb0), eb1 = ex2(yb1);
+                                const uint64_t ea2 = pack2(ea0, ea1), eb2 = pack2(eb0, eb1);
+                                za2 = add2(za2, ea2);
+                                zb2 = add2(zb2, eb2);
+                                if constexpr (DIV == FSD_DIV_JS) {
+                                    sa2 = fma2(ea2, ya2, sa2);
+                                    sb2 = fma2(eb2, yb2, sb2);
+                                }
+                                if constexpr (DIV == FSD_DIV_KL) {
+                                    if (ea0 > 0.f) kk = fmaf(ea0, ya0 - yb0, kk);
+                                    if (ea1 > 0.f) kk = fmaf(ea1, ya1 - yb1, kk);
+                                }
+                                e[v][j] = ea0; e[v][j + 1] = ea1;
+                                e[v][EPV + j] = eb0; e[v][EPV + j + 1] = eb1;
+                            }
                         } else {
 #pragma unroll
-                            for (int j = 0; j < EPT; ++j) ereg[(s - NT < 0 ? 0 : s - NT) * EPT + j] = e[j];
+                            for (int j = 0; j < EPT; ++j) e[v][j] = 0.f;
+                        }
+                    }
+                    if constexpr (kSecondSweep) {
+#pragma unroll
+                        for (int v = 0; v < VPT; ++v) {
+                            if (s < NT) {
+                                tmem_st<EPT>(taddr + (s * VPT + v) * EPT, e[v]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < EPT; ++j) ereg[(s - NT < 0 ? 0 : s - NT) * EPS + v * EPT + j] = e[v][j];
+                            }
                         }
                     }
                     // this warp is done with the slot; the last warp to say so refills it
                     __syncwarp();
                     if (lane == 0) {
-                        if (atom_add_acq_rel(&sh.readers_done[slot], 1) == kStreamWarps - 1) {
+                        if (atom_add_relaxed(&sh.readers_done[slot], 1) == kStreamWarps - 1) {
                             sh.readers_done[slot] = 0;
                             issue_stage(gs + kRing);
                         }
                     }
-                    __syncwarp();
                 }
             }
             if constexpr (kSecondSweep) tmem_wait_st();
 
             // thread -> warp: bring the sums to the warp's reference (exact power-of-two factors)
-            const float za = sum2(za2), zb = sum2(zb2), sa = sum2(sa2), sb = sum2(sb2);
+            const float za = sum2(za2), zb = sum2(zb2);
             const float wka = warp_max_nan(ka), wkb = warp_max_nan(kb);
             const float da = ka == -INFINITY ? 0.f : ka - wka, db = kb == -INFINITY ? 0.f : kb - wkb;
             const float fa = ka == -INFINITY ? 0.f : pow2_int(da), fb = kb == -INFINITY ? 0.f : pow2_int(db);
             float v_za = za * fa, v_zb = zb * fb;
-            float v_sa = fa * fmaf(da, za, sa), v_sb = fb * fmaf(db, zb, sb);
-            float v_kk = fa * fmaf(da - db, za, kk);
+            float v_s0 = 0.f, v_sb = 0.f;
+            if constexpr (DIV == FSD_DIV_JS) { v_s0 = fa * fmaf(da, za, sum2(sa2)); v_sb = fb * fmaf(db, zb, sum2(sb2)); }
+            if constexpr (DIV == FSD_DIV_KL) v_s0 = scale_kl(fa, fmaf(da - db, za, kk));
 #pragma unroll
             for (int m = 16; m > 0; m >>= 1) {
                 v_za += __shfl_xor_sync(0xffffffffu, v_za, m);
                 v_zb += __shfl_xor_sync(0xffffffffu, v_zb, m);
-                if constexpr (DIV == FSD_DIV_JS) {
-                    v_sa += __shfl_xor_sync(0xffffffffu, v_sa, m);
-                    v_sb += __shfl_xor_sync(0xffffffffu, v_sb, m);
-                }
-                if constexpr (DIV == FSD_DIV_KL) v_kk += __shfl_xor_sync(0xffffffffu, v_kk, m);
+                if constexpr (DIV != FSD_DIV_TV) v_s0 += __shfl_xor_sync(0xffffffffu, v_s0, m);
+                if constexpr (DIV == FSD_DIV_JS) v_sb += __shfl_xor_sync(0xffffffffu, v_sb, m);
             }
-            mine.ka = wka; mine.kb = wkb; mine.za = v_za; mine.zb = v_zb; mine.sa = v_sa; mine.sb = v_sb; mine.kk = v_kk;
+            mine.ka = wka; mine.kb = wkb; mine.za = v_za; mine.zb = v_zb; mine.s0 = v_s0; mine.sb = v_sb;
             mine.diff = __reduce_or_sync(0xffffffffu, diff);
         }
         mine.x = x_carry;
 
-        // ---- post the warp's statistics; the last warp of the CTA to do so combines them and
-        //      delivers the CTA's statistics to every CTA of the cluster (itself included) ----
-        int last = 0;
-        if (lane == 0) {
-            sh.ws[par][warp] = mine;
-            last = atom_add_acq_rel(&sh.stats_done[par], 1) == kStreamWarps - 1;
-            if (last) sh.stats_done[par] = 0;
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-            PartStats w;
-            w.ka = -INFINITY; w.kb = -INFINITY; w.za = 0.f; w.zb = 0.f; w.sa = 0.f; w.sb = 0.f; w.kk = 0.f; w.x = 0.f; w.diff = 0;
-            if (lane < kStreamWarps) w = sh.ws[par][lane];
-            PartStats c;
+        // ---- exchange.  Every warp leaves its statistics in shared memory and counts itself in
+        //      on a named barrier; this round's combiner warp waits there for the others, folds
+        //      the warps' statistics, sends the CTA's to every CTA of the cluster (itself
+        //      included), waits for all of the cluster's to land, folds those and leaves the
+        //      totals for the CTA.  Only the combiner polls; everyone else sleeps on a barrier. ----
+        if (lane == 0) sh.ws[warp] = mine;
+        __syncwarp();
+        if (warp != static_cast<int>(li & (kStreamWarps - 1))) {
+            __threadfence_block();
+            named_arrive(kBarPosted);
+        } else {
+            named_sync(kBarPosted);
+            Stats w;
+            w.ka = -INFINITY; w.kb = -INFINITY; w.za = 0.f; w.zb = 0.f; w.s0 = 0.f; w.sb = 0.f; w.x = 0.f; w.diff = 0;
+            if (lane < kStreamWarps) w = sh.ws[lane];
+            Stats c;
             c.ka = warp_max_nan(w.ka); c.kb = warp_max_nan(w.kb);
-            const float da = w.ka == -INFINITY ? 0.f : w.ka - c.ka, db = w.kb == -INFINITY ? 0.f : w.kb - c.kb;
-            const float fa = w.ka == -INFINITY ? 0.f : pow2_int(da), fb = w.kb == -INFINITY ? 0.f : pow2_int(db);
-            c.za = w.za * fa; c.zb = w.zb * fb;
-            c.sa = fa * fmaf(da, w.za, w.sa); c.sb = fb * fmaf(db, w.zb, w.sb);
-            c.kk = fa * fmaf(da - db, w.za, w.kk);
-            c.x = w.x;
+            {
+                const float da = w.ka == -INFINITY ? 0.f : w.ka - c.ka, db = w.kb == -INFINITY ? 0.f : w.kb - c.kb;
+                const float fa = w.ka == -INFINITY ? 0.f : pow2_int(da), fb = w.kb == -INFINITY ? 0.f : pow2_int(db);
+                c.za = w.za * fa; c.zb = w.zb * fb;
+                c.s0 = DIV == FSD_DIV_KL ? scale_kl(fa, fmaf(da - db, w.za, w.s0)) : fa * fmaf(da, w.za, w.s0);
+                c.sb = fb * fmaf(db, w.zb, w.sb);
+                c.x = w.x;
+            }
 #pragma unroll
             for (int m = 8; m > 0; m >>= 1) {
                 c.za += __shfl_xor_sync(0xffffffffu, c.za, m); c.zb += __shfl_xor_sync(0xffffffffu, c.zb, m);
-                c.sa += __shfl_xor_sync(0xffffffffu, c.sa, m); c.sb += __shfl_xor_sync(0xffffffffu, c.sb, m);
-                c.kk += __shfl_xor_sync(0xffffffffu, c.kk, m); c.x += __shfl_xor_sync(0xffffffffu, c.x, m);
+                c.s0 += __shfl_xor_sync(0xffffffffu, c.s0, m); c.sb += __shfl_xor_sync(0xffffffffu, c.sb, m);
+                c.x += __shfl_xor_sync(0xffffffffu, c.x, m);
             }
             c.diff = __reduce_or_sync(0xffffffffu, w.diff);
-            if (lane < C) {                                // lanes 0..15 hold the totals; lane r serves CTA r
-                cluster.map_shared_rank(&sh, lane)->xch[par][rank] = c;
-                mbar_arrive_remote(&sh.xbar[par], static_cast<uint32_t>(lane));
+            if (lane == 0) mbar_arrive_expect_tx(&sh.xbar[par], static_cast<uint32_t>(C) * sizeof(Stats));
+            if (lane < C) {                                // lanes 0..15 hold the CTA's statistics; lane r serves CTA r
+                Stats* dst = &sh.xch[par][rank];
+                st_async_remote(dst, &sh.xbar[par], static_cast<uint32_t>(lane), c.ka, c.kb, c.za, c.zb);
+                st_async_remote(&dst->s0, &sh.xbar[par], static_cast<uint32_t>(lane), c.s0, c.sb, c.x, __uint_as_float(c.diff));
             }
-        }
-        __syncwarp();
-
-        // ---- meanwhile: sweep A of the next pair ----
-        const int next = item + n_clusters;
-        float ra_n = -INFINITY, rb_n = -INFINITY;
-        uint32_t diff_n = 0;
-        if (live && next < P.n_items) sweep_a(g + ns, ra_n, rb_n, diff_n);
-
-        // ---- cluster totals: every CTA's statistics have arrived in this CTA's shared memory ----
-        mbar_wait_cluster(&sh.xbar[par], xphase, P.timeout_flag, dead);
-        float Ka, Kb, tZa, tZb;
-        {
-            PartStats c;
-            c.ka = -INFINITY; c.kb = -INFINITY; c.za = 0.f; c.zb = 0.f; c.sa = 0.f; c.sb = 0.f; c.kk = 0.f; c.x = 0.f; c.diff = 0;
-            if (lane < C) c = sh.xch[par][lane];
-            Ka = warp_max_nan(c.ka); Kb = warp_max_nan(c.kb);
-            const float da = c.ka == -INFINITY ? 0.f : c.ka - Ka, db = c.kb == -INFINITY ? 0.f : c.kb - Kb;
-            const float fa = c.ka == -INFINITY ? 0.f : pow2_int(da), fb = c.kb == -INFINITY ? 0.f : pow2_int(db);
-            tZa = c.za * fa; tZb = c.zb * fb;
+            mbar_wait_cluster(&sh.xbar[par], xphase, P.timeout_flag, dead);
+            // cluster totals for the second sweep (float is enough there); lane r holds CTA r's part
+            Stats t;
+            t.ka = -INFINITY; t.kb = -INFINITY; t.za = 0.f; t.zb = 0.f; t.s0 = 0.f; t.sb = 0.f; t.x = 0.f; t.diff = 0;
+            if (lane < C) t = sh.xch[par][lane];
+            const float Ka = warp_max_nan(t.ka), Kb = warp_max_nan(t.kb);
+            float tza = t.ka == -INFINITY ? 0.f : t.za * pow2_int(t.ka - Ka);
+            float tzb = t.kb == -INFINITY ? 0.f : t.zb * pow2_int(t.kb - Kb);
 #pragma unroll
-            for (int m = 4; m > 0; m >>= 1) {
-                tZa += __shfl_xor_sync(0xffffffffu, tZa, m); tZb += __shfl_xor_sync(0xffffffffu, tZb, m);
+            for (int m = 8; m > 0; m >>= 1) {
+                tza += __shfl_xor_sync(0xffffffffu, tza, m); tzb += __shfl_xor_sync(0xffffffffu, tzb, m);
             }
-            tZa = __shfl_sync(0xffffffffu, tZa, 0);
-            tZb = __shfl_sync(0xffffffffu, tZb, 0);
-            // one warp of rank 0: all totals in double, into the pair's record; the previous pair
-            // gets its second-sweep sum
-            if (rank == 0 && warp == kStreamWarps - 1) {
-                double dza = 0, dzb = 0, dsa = 0, dsb = 0, dkk = 0, dx = 0;
-                if (lane < C) {
-                    const double ffa = fa, ffb = fb;
-                    dza = static_cast<double>(c.za) * ffa; dzb = static_cast<double>(c.zb) * ffb;
-                    dsa = ffa * (static_cast<double>(c.sa) + static_cast<double>(da) * c.za);
-                    dsb = ffb * (static_cast<double>(c.sb) + static_cast<double>(db) * c.zb);
-                    dkk = ffa * (static_cast<double>(c.kk) + static_cast<double>(da - db) * c.za);
-                    dx = c.x;
-                }
-#pragma unroll
-                for (int m = 4; m > 0; m >>= 1) {
-                    dza += shfl_xor_d(dza, m); dzb += shfl_xor_d(dzb, m); dsa += shfl_xor_d(dsa, m);
-                    dsb += shfl_xor_d(dsb, m); dkk += shfl_xor_d(dkk, m); dx += shfl_xor_d(dx, m);
-                }
-                const uint32_t edf = __reduce_or_sync(0xffffffffu, c.diff);
-                if (lane == 0) {
-                    if (prev_item >= 0) P.records[prev_item].X = dx;
-                    if (live) {
-                        PairRecord r;
-                        r.Za = dza; r.Zb = dzb; r.Sa = dsa; r.Sb = dsb; r.K = dkk; r.X = 0.0;
-                        r.ka = Ka; r.kb = Kb; r.differ = edf; r.state = bad ? kRecordBadTree : kRecordStats;
-                        P.records[item] = r;
-                    }
+            if (lane == 0) *reinterpret_cast<float4*>(sh.tot) = make_float4(Ka, Kb, tza, tzb);
+            named_sync(kBarTotals);
+            // rank 0 hands the parts to the finish kernel, which folds them in double; the
+            // previous pair gets its second-sweep sums
+            if (rank == 0 && lane < C) {
+                if (prev_item >= 0) P.records[prev_item].x[lane] = t.x;
+                if (live) {
+                    PairRecord* r = P.records + item;
+                    r->part[lane] = t;
+                    if (lane == 0) { r->ncta = static_cast<uint32_t>(C); r->state = bad ? kRecordBadTree : kRecordStats; }
                 }
             }
         }
+        if (warp != static_cast<int>(li & (kStreamWarps - 1))) named_sync(kBarTotals);
+        const float4 tot = *reinterpret_cast<const float4*>(sh.tot);
+        const float Ka = tot.x, Kb = tot.y, tZa = tot.z, tZb = tot.w;
         prev_item = -1;
         x_carry = 0.f;
         if (!live) break;
@@ -579,28 +671,35 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
 #pragma unroll
             for (int s = 0; s < kMaxStagesPerPair; ++s) {
                 if (s < ns) {
-                    float e[EPT];
+                    float e[VPT][EPT];
                     if (s < NT) {
-                        tmem_ld<EPT>(taddr + s * EPT, e);
+#pragma unroll
+                        for (int v = 0; v < VPT; ++v) tmem_ld<EPT>(taddr + (s * VPT + v) * EPT, e[v]);
                         tmem_wait_ld();
                     } else {
 #pragma unroll
-                        for (int j = 0; j < EPT; ++j) e[j] = ereg[(s - NT < 0 ? 0 : s - NT) * EPT + j];
+                        for (int v = 0; v < VPT; ++v) {
+#pragma unroll
+                            for (int j = 0; j < EPT; ++j) e[v][j] = ereg[(s - NT < 0 ? 0 : s - NT) * EPS + v * EPT + j];
+                        }
                     }
 #pragma unroll
-                    for (int j = 0; j < EPV; j += 2) {
-                        const uint64_t ea2 = pack2(e[j], e[j + 1]), eb2 = pack2(e[EPV + j], e[EPV + j + 1]);
-                        if constexpr (DIV == FSD_DIV_JS) {
-                            const uint64_t s2 = fma2(eb2, ib2, fma2(ea2, ia2, tiny2));
-                            float s0, s1;
-                            unpack2(s2, s0, s1);
-                            x2 = fma2(s2, pack2(lg2(s0), lg2(s1)), x2);
-                        } else {
-                            // separately rounded products: a fused p - q would make TV(p, p) != 0
-                            const uint64_t d2 = fma2(mul2(eb2, ib2), pack2(-1.f, -1.f), mul2(ea2, ia2));
-                            float d0, d1;
-                            unpack2(d2, d0, d1);
-                            xt += fabsf(d0) + fabsf(d1);
+                    for (int v = 0; v < VPT; ++v) {
+#pragma unroll
+                        for (int j = 0; j < EPV; j += 2) {
+                            const uint64_t ea2 = pack2(e[v][j], e[v][j + 1]), eb2 = pack2(e[v][EPV + j], e[v][EPV + j + 1]);
+                            if constexpr (DIV == FSD_DIV_JS) {
+                                const uint64_t s2 = fma2(eb2, ib2, fma2(ea2, ia2, tiny2));
+                                float s0, s1;
+                                unpack2(s2, s0, s1);
+                                x2 = fma2(s2, pack2(lg2(s0), lg2(s1)), x2);
+                            } else {
+                                // separately rounded products: a fused p - q would make TV(p, p) != 0
+                                const uint64_t d2 = fma2(mul2(eb2, ib2), pack2(-1.f, -1.f), mul2(ea2, ia2));
+                                float d0, d1;
+                                unpack2(d2, d0, d1);
+                                xt += fabsf(d0) + fabsf(d1);
+                            }
                         }
                     }
                 }
@@ -614,8 +713,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
         // ---- next pair ----
         g += ns;
         ++li;
-        item = next;
-        ra = ra_n; rb = rb_n; diff = diff_n;
+        item += n_clusters;
     }
 
     // ---- release tensor memory ----
@@ -632,7 +730,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) fsd_pair_stream_kernel(Stre
 // per SM for any kernel that allocates tensor memory (it cannot know how many columns); the
 // streaming kernel allocates half of an SM's tensor memory, so two CTAs do fit, and the grid
 // is sized from this twin instead.
-__global__ void __launch_bounds__(kStreamThreads, 2) fsd_stream_occupancy_twin(int* p) {
+__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_stream_occupancy_twin(int* p) {
     extern __shared__ unsigned char smem_raw[];
     if (p != nullptr) p[threadIdx.x] = smem_raw[threadIdx.x];
 }

@@ -146,6 +146,33 @@ def test_nonfinite_rows_are_flagged_not_propagated():
     _check(c, mode="sd")
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_wide_dynamic_range_moves_the_reference(dtype):
+    """Rows whose largest logits come late and far above the first ones (masked prefixes, late
+    spikes, steep ramps): whatever reference a streaming softmax starts from has to move."""
+    B, gamma, V = 4, 3, 40000
+    c = gi.make_chain(B, gamma, V, dtype=dtype, recipe="spike", sigma=(0.5, 1.0), workload_id=306)
+    f32 = dtype == "f32"
+    t = c.target if f32 else gi.bf16_bits_to_f32(c.target)
+    d = c.draft if f32 else gi.bf16_bits_to_f32(c.draft)
+    k = np.arange(V, dtype=np.float32)
+    t[0, :, :9000] = -np.inf                      # nothing finite for the first stages
+    d[0, :, :13000] = -np.inf
+    t[1, :, 30011:30014] += 90.0                  # late spikes: 130 binades above the rest
+    d[1, :, 39990:] += 75.0
+    t[2] += (k * 0.01 - 200.0)                    # +-200 nats ramp: the reference moves again and again
+    d[2] += (k * 0.0125 - 250.0)
+    t[3] -= k * 0.01                              # falling ramp: the first reference stays
+    d[3, :, 1::2] = -np.inf
+    d[3, :, -1] = 300.0                           # and one jump of > 126 binades at the very end
+    if not f32:
+        c.target[:] = gi.f32_to_bf16_bits(t)
+        c.draft[:] = gi.f32_to_bf16_bits(d)
+    for div in ("js", "kl", "tv"):
+        _check(c, div=div, T=0.3)
+    _check(c, mode="rfsd", T=0.3)
+
+
 def test_uniform_extremes_for_sampling():
     c = gi.make_chain(6, 2, 5000, dtype="bf16", recipe="zipf", sigma=(0.5,), workload_id=303)
     c.u_sample[:] = np.array([0.0, np.nextafter(np.float32(1), np.float32(0)), 0.5, 1e-7, 0.999, 0.25], np.float32)
