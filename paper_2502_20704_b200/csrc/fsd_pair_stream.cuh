@@ -267,16 +267,6 @@ __device__ __forceinline__ void named_sync(int id) {
 }
 constexpr int kBarPosted = 1, kBarTotals = 2;
 
-// Shared-memory counter increment, returns the old value.  Relaxed: a warp's reads of a ring
-// slot have completed by the time it counts itself out (their values were consumed), and the
-// thread that refills the slot orders its own reset of the counter before the copy through the
-// proxy fence and the barrier it arms.
-__device__ __forceinline__ int atom_add_relaxed(int* p, int v) {
-    int old;
-    asm volatile("atom.relaxed.cta.shared::cta.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
-    return old;
-}
-
 // ---- cluster-scope mbarrier wait (the statistics exchange) ------------------------------------
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -301,7 +291,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
 struct StreamShared {
     uint64_t full[kRing];      // a ring stage has landed
     uint64_t xbar[2];          // all CTAs' statistics have landed here (per parity): 1 arrival + C * 32 bytes
-    int readers_done[kRing];   // warps that have finished reading the slot's current stage
+    uint64_t empty[kRing];     // every warp has finished reading the slot's current stage
     uint32_t tmem_base;
     alignas(16) float tot[4];  // cluster totals of the current pair: Ka, Kb, Za, Zb
     Stats ws[kStreamWarps];    // the warps' statistics of the current pair
@@ -340,7 +330,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     // ---- set-up: barriers, tensor memory ----
     if (blockIdx.x == 0 && tid == 0) *P.timeout_flag = 0;   // a wait needs far longer to run out than this store takes
     if (tid == 0) {
-        for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); sh.readers_done[s] = 0; }
+        for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kStreamWarps); }
         mbar_init(&sh.xbar[0], 1); mbar_init(&sh.xbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -554,12 +544,15 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
                             }
                         }
                     }
-                    // this warp is done with the slot; the last warp to say so refills it
+                    // This warp is done with the slot.  Nobody waits for the slot to drain: one stage
+                    // later, when every warp has long left it, this stage's duty warp refills it.
                     __syncwarp();
                     if (lane == 0) {
-                        if (atom_add_relaxed(&sh.readers_done[slot], 1) == kStreamWarps - 1) {
-                            sh.readers_done[slot] = 0;
-                            issue_stage(gs + kRing);
+                        mbar_arrive(&sh.empty[slot]);
+                        if (gs > 0 && warp == static_cast<int>(gs % kStreamWarps)) {
+                            const uint32_t ps = gs - 1;
+                            mbar_wait(&sh.empty[ps % kRing], (ps / kRing) & 1, P.timeout_flag, dead);
+                            issue_stage(ps + kRing);
                         }
                     }
                 }
