@@ -409,16 +409,31 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             if (lane == 0 && lp >= 0) atomicMax(&sh.last_pos, lp);
             __syncthreads();
             if (tid == 0) P.next_token[b] = sh.last_pos;
-        } else if (tid == c) {
-            double running = excl;
-            int tok = -1, lastp = -1;
-            for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int k, float xa, float) {
-                const double w = exp2_table(fma(static_cast<double>(xa), kLog2eD, -kref), tab);
-                running += w;
+        } else if (warp == (c >> 5)) {
+            // the warp of the thread whose chunk holds the crossing walks that chunk together:
+            // 32 weights at a time, prefix sums in index order
+            const int src = c & 31;
+            const int ck0 = __shfl_sync(0xffffffffu, k0, src), ck1 = __shfl_sync(0xffffffffu, k1, src);
+            double base = __shfl_sync(0xffffffffu, excl, src);
+            int tok = 0x7fffffff, lastp = -1;
+            for (int kb = ck0; kb < ck1; kb += 32) {
+                const int k = kb + lane;
+                double w = 0.0;
+                if (k < ck1) w = exp2_table(fma(static_cast<double>(load_logit<DT>(a_row, k)), kLog2eD, -kref), tab);
+                double run = w;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const double up = __shfl_up_sync(0xffffffffu, run, d);
+                    if (lane >= d) run += up;
+                }
+                run += base;
                 if (w > 0.0) lastp = k;
-                if (tok < 0 && running > t_local) tok = k;
-            });
-            P.next_token[b] = tok >= 0 ? tok : lastp;
+                if (w > 0.0 && run > t_local && k < tok) tok = k;
+                base = __shfl_sync(0xffffffffu, run, 31);
+            }
+            tok = __reduce_min_sync(0xffffffffu, tok);
+            lastp = __reduce_max_sync(0xffffffffu, lastp);
+            if (lane == 0) P.next_token[b] = tok != 0x7fffffff ? tok : lastp;
         }
         return;
     }
