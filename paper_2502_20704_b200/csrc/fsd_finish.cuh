@@ -121,44 +121,62 @@ struct PairTotals {
     float ka, kb;
     uint32_t differ;
 };
-__device__ inline PairTotals fold_record(const PairRecord& rec, int div) {
+// 2^d for an integer-valued d <= 0, exact; 0 below the normal range
+__device__ __forceinline__ double pow2_int_d(double d) {
+    return d < -1022.0 ? 0.0 : __hiloint2double((1023 + static_cast<int>(d)) << 20, 0);
+}
+__device__ __forceinline__ double group8_sum(double v) {
+#pragma unroll
+    for (int m = 4; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+    return v;
+}
+// Called by all 32 lanes: lane 8*q + r folds part r of the record `rec` of group q (null: no
+// record for this group); every lane of a group returns the group's totals.
+__device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
+    const int r = threadIdx.x & 7;
     PairTotals t;
-    t.Za = 0.0; t.Zb = 0.0; t.Sa = 0.0; t.Sb = 0.0; t.K = 0.0; t.X = 0.0; t.differ = 0;
-    const int n = static_cast<int>(rec.ncta) < kStreamMaxCluster ? static_cast<int>(rec.ncta) : kStreamMaxCluster;
-    float ka = -INFINITY, kb = -INFINITY;
-    for (int r = 0; r < n; ++r) {                       // NaN references win
-        const float a = rec.part[r].ka, b = rec.part[r].kb;
-        ka = (a != a || ka != ka) ? __int_as_float(0x7fc00000) : fmaxf(ka, a);
-        kb = (b != b || kb != kb) ? __int_as_float(0x7fc00000) : fmaxf(kb, b);
+    Stats c;
+    c.ka = -INFINITY; c.kb = -INFINITY; c.za = 0.f; c.zb = 0.f; c.s0 = 0.f; c.sb = 0.f; c.x = 0.f; c.diff = 0;
+    float x = 0.f;
+    if (rec != nullptr && r < static_cast<int>(rec->ncta)) { c = rec->part[r]; x = rec->x[r]; }
+    float ka = c.ka, kb = c.kb;                          // NaN references win
+#pragma unroll
+    for (int m = 4; m > 0; m >>= 1) {
+        const float oa = __shfl_xor_sync(0xffffffffu, ka, m), ob = __shfl_xor_sync(0xffffffffu, kb, m);
+        ka = (oa != oa || ka != ka) ? __int_as_float(0x7fc00000) : fmaxf(ka, oa);
+        kb = (ob != ob || kb != kb) ? __int_as_float(0x7fc00000) : fmaxf(kb, ob);
     }
     t.ka = ka; t.kb = kb;
-    for (int r = 0; r < n; ++r) {
-        const Stats c = rec.part[r];
-        const double da = c.ka == -INFINITY ? 0.0 : static_cast<double>(c.ka) - ka;
-        const double db = c.kb == -INFINITY ? 0.0 : static_cast<double>(c.kb) - kb;
-        const double fa = c.ka == -INFINITY ? 0.0 : (da < -2000.0 ? 0.0 : scalbn(1.0, static_cast<int>(da)));
-        const double fb = c.kb == -INFINITY ? 0.0 : (db < -2000.0 ? 0.0 : scalbn(1.0, static_cast<int>(db)));
-        t.Za += fa * c.za; t.Zb += fb * c.zb;
-        if (div == FSD_DIV_KL) {
-            t.K += c.s0 == INFINITY ? static_cast<double>(INFINITY) : fa * (static_cast<double>(c.s0) + (da - db) * c.za);
-        } else {
-            t.Sa += fa * (static_cast<double>(c.s0) + da * c.za);
-            t.Sb += fb * (static_cast<double>(c.sb) + db * c.zb);
-        }
-        t.X += rec.x[r];
-        t.differ |= c.diff;
+    const double da = c.ka == -INFINITY ? 0.0 : static_cast<double>(c.ka) - ka;
+    const double db = c.kb == -INFINITY ? 0.0 : static_cast<double>(c.kb) - kb;
+    const double fa = (c.ka == -INFINITY || da != da) ? 0.0 : pow2_int_d(da);
+    const double fb = (c.kb == -INFINITY || db != db) ? 0.0 : pow2_int_d(db);
+    t.Za = group8_sum(fa * c.za); t.Zb = group8_sum(fb * c.zb);
+    t.Sa = 0.0; t.Sb = 0.0; t.K = 0.0;
+    if (div == FSD_DIV_KL) {
+        const bool inf = c.s0 == INFINITY;
+        const double k = inf ? 0.0 : fa * (static_cast<double>(c.s0) + (da - db) * c.za);
+        t.K = group8_sum(k);
+        const unsigned any_inf = __ballot_sync(0xffffffffu, inf) >> (threadIdx.x & 24) & 0xffu;
+        if (any_inf) t.K = static_cast<double>(INFINITY);
+    } else {
+        t.Sa = group8_sum(fa * (static_cast<double>(c.s0) + da * c.za));
+        t.Sb = group8_sum(fb * (static_cast<double>(c.sb) + db * c.zb));
     }
+    t.X = group8_sum(static_cast<double>(x));
+    uint32_t df = c.diff;
+#pragma unroll
+    for (int m = 4; m > 0; m >>= 1) df |= __shfl_xor_sync(0xffffffffu, df, m);
+    t.differ = df;
     return t;
 }
 
-__device__ inline void judge_record(const FinishParams& P, int item, const void* a_row, const void* b_row, int dt,
+__device__ inline void judge_record(const FinishParams& P, int item, const PairTotals& r, const void* a_row, const void* b_row, int dt,
                                     float& D_out, int& bit_out, int& st_out) {
-    const PairRecord& rec = P.records[item];
-    if (rec.state & kRecordBadTree) {
+    if (P.records[item].state & kRecordBadTree) {
         D_out = __int_as_float(0x7fc00000); bit_out = 0; st_out = FSD_ROW_BADTREE;
         return;
     }
-    const PairTotals r = fold_record(rec, P.div);
     const bool finite = isfinite(r.ka) && isfinite(r.kb) && r.Za > 0.0 && r.Zb > 0.0 && isfinite(r.Za) && isfinite(r.Zb);
     float D = __int_as_float(0x7fc00000);
     if (finite) D = r.differ ? static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X)) : 0.0f;
@@ -232,25 +250,35 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
 
     // ---- 1. divergences, accept bits, status of this row's pairs ----
     int st = 0, first = G;
-    for (int i = tid; i < G; i += blockDim.x) {
-        const int item = b * G + i;
-        int bit, s;
-        if (P.records != nullptr) {
-            int trow = i;
-            if (tree) {
-                const int par = P.parent[item];
-                trow = (par >= -1 && par < i) ? par + 1 : 0;
+    if (P.records != nullptr) {
+        // four pairs per warp: eight lanes fold a pair's record, the first of them judges it
+        for (int i0 = 4 * warp; i0 < G; i0 += 4 * (blockDim.x >> 5)) {
+            const int i = i0 + (lane >> 3);
+            const int item = b * G + i;
+            const PairTotals tot = fold_record(i < G ? P.records + item : nullptr, P.div);
+            if (i < G && (lane & 7) == 0) {
+                int trow = i;
+                if (tree) {
+                    const int par = P.parent[item];
+                    trow = (par >= -1 && par < i) ? par + 1 : 0;
+                }
+                float D;
+                int bit, s;
+                judge_record(P, item, tot, t_base + static_cast<size_t>(trow) * rb, d_base + static_cast<size_t>(i) * rb, DT, D, bit, s);
+                if (rank == 0) P.divergence[item] = D;
+                st |= s;
+                if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
+                else if (!bit && i < first) first = i;
             }
-            float D;
-            judge_record(P, item, t_base + static_cast<size_t>(trow) * rb, d_base + static_cast<size_t>(i) * rb, DT, D, bit, s);
-            if (rank == 0) P.divergence[item] = D;
-        } else {
-            bit = P.item_bits[item];
-            s = P.item_status[item];
         }
-        st |= s;
-        if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
-        else if (!bit && i < first) first = i;
+    } else {
+        for (int i = tid; i < G; i += blockDim.x) {
+            const int item = b * G + i;
+            const int bit = P.item_bits[item];
+            st |= P.item_status[item];
+            if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
+            else if (!bit && i < first) first = i;
+        }
     }
     if (tid == 0 && P.timeout_flag != nullptr && *P.timeout_flag != 0) st |= FSD_ROW_TIMEOUT;
     st = __reduce_or_sync(0xffffffffu, st);
