@@ -141,7 +141,9 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Pair
     if (C > 0) {
         StreamParams sp;
         sp.target = pp.target; sp.draft = pp.draft; sp.parent = pp.parent; sp.B = pp.B; sp.G = pp.G;
-        sp.nvec_row = nvec_row; sp.n_items = items; sp.records = records; sp.timeout_flag = flags;
+        sp.nvec_row = nvec_row; sp.n_items = items; sp.records = records; sp.timeout_flag = flags; sp.next_pair = flags + 1;
+        // the flag block starts every call at zero: [0] timeout, [1] pairs handed out
+        if (cudaMemsetAsync(flags, 0, kAlign, s) != cudaSuccess) return FSD_ERR_CUDA;
         int rc;
         if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, C, s);
         else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, C, s);

@@ -82,7 +82,8 @@ struct StreamParams {
     int nvec_row;              // 16-byte vectors per logit row
     int n_items;               // B * G
     PairRecord* records;       // [B * G]
-    int* timeout_flag;         // set to 1 if a bounded wait ran out
+    int* timeout_flag;         // set to 1 if a bounded wait ran out; zero at launch
+    int* next_pair;            // pairs handed out beyond each cluster's fixed first ones; zero at launch
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -293,6 +294,7 @@ struct StreamShared {
     uint64_t xbar[2];          // all CTAs' statistics have landed here (per parity): 1 arrival + C * 32 bytes
     uint64_t empty[kRing];     // every warp has finished reading the slot's current stage
     uint32_t tmem_base;
+    int items[8];              // pair ids of this cluster's rounds, indexed by round & 7
     alignas(16) float tot[4];  // cluster totals of the current pair: Ka, Kb, Za, Zb
     Stats ws[kStreamWarps];    // the warps' statistics of the current pair
     Stats xch[2][kStreamMaxCluster];         // written by the peers (and by this CTA for its own rank)
@@ -328,8 +330,13 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     const size_t row_bytes = static_cast<size_t>(P.nvec_row) * 16;
 
     // ---- set-up: barriers, tensor memory ----
-    if (blockIdx.x == 0 && tid == 0) *P.timeout_flag = 0;   // a wait needs far longer to run out than this store takes
+    // A cluster's first `ahead` pairs are fixed (cluster_id + round * n_clusters): that is as far
+    // as the ring reads ahead.  Every later pair is the next one nobody has taken yet, claimed
+    // `ahead` rounds early by rank 0 and sent round with that round's statistics, so clusters
+    // that happen to run faster take more pairs and all finish together.
+    const int ahead = 2 + (kRing - 2) / ns;
     if (tid == 0) {
+        for (int k = 0; k < ahead; ++k) sh.items[k] = cluster_id + k * n_clusters;
         for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kStreamWarps); }
         mbar_init(&sh.xbar[0], 1); mbar_init(&sh.xbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -353,9 +360,9 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     // copies are issued as early as possible and the work is spread over the warps.
     auto issue_stage = [&](uint32_t gg) {
         const uint32_t k = gg / static_cast<uint32_t>(ns), s = gg - k * static_cast<uint32_t>(ns);
-        const long long item = cluster_id + static_cast<long long>(k) * n_clusters;
+        const int item = sh.items[k & 7];
         if (item >= P.n_items) return;
-        const int b = static_cast<int>(item / P.G), i = static_cast<int>(item - static_cast<long long>(b) * P.G);
+        const int b = item / P.G, i = item - b * P.G;
         int trow = i;
         if (P.parent != nullptr) {
             const int par = __ldg(P.parent + item);
@@ -384,12 +391,18 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     float x_carry = 0.f;                             // previous pair's second-sweep sum of this warp
     int prev_item = -1;                              // pair whose second-sweep sum is still to be published
     int item = cluster_id;
+    uint32_t claimed = 0;                            // rank 0, combiner lane 0: the pair id taken this round
 
     for (;;) {
         const bool live = item < P.n_items;          // one extra round publishes the last pair's second sweep
         if (!live && prev_item < 0) break;
         const int par = static_cast<int>(li & 1);
         const uint32_t xphase = (li >> 1) & 1;
+        if (rank == 0 && lane == 0 && warp == static_cast<int>(li & (kStreamWarps - 1))) {
+            // asked now, needed only when the statistics go out
+            const long long id = static_cast<long long>(ahead) * n_clusters + atomicAdd(P.next_pair, 1);
+            claimed = id < 0x3fffffffLL ? static_cast<uint32_t>(id) : 0x3fffffffu;
+        }
         bool bad = false;
         if (live && P.parent != nullptr) {
             const int i = item % P.G;
@@ -611,7 +624,11 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
                 c.s0 += __shfl_xor_sync(0xffffffffu, c.s0, m); c.sb += __shfl_xor_sync(0xffffffffu, c.sb, m);
                 c.x += __shfl_xor_sync(0xffffffffu, c.x, m);
             }
-            c.diff = __reduce_or_sync(0xffffffffu, w.diff);
+            c.diff = __reduce_or_sync(0xffffffffu, w.diff) != 0 ? 1u : 0u;
+            {
+                const uint32_t cl = __shfl_sync(0xffffffffu, claimed, 0);   // rank 0's message carries the pair id it took
+                if (rank == 0) c.diff |= cl << 1;
+            }
             if (lane == 0) mbar_arrive_expect_tx(&sh.xbar[par], static_cast<uint32_t>(C) * sizeof(Stats));
             if (lane < C) {                                // lanes 0..15 hold the CTA's statistics; lane r serves CTA r
                 Stats* dst = &sh.xch[par][rank];
@@ -623,6 +640,11 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
             Stats t;
             t.ka = -INFINITY; t.kb = -INFINITY; t.za = 0.f; t.zb = 0.f; t.s0 = 0.f; t.sb = 0.f; t.x = 0.f; t.diff = 0;
             if (lane < C) t = sh.xch[par][lane];
+            {
+                const uint32_t nxt = __shfl_sync(0xffffffffu, t.diff, 0) >> 1;
+                t.diff &= 1u;
+                if (lane == 0) sh.items[(li + ahead) & 7] = static_cast<int>(nxt);
+            }
             const float Ka = warp_max_nan(t.ka), Kb = warp_max_nan(t.kb);
             float tza = t.ka == -INFINITY ? 0.f : t.za * pow2_int(t.ka - Ka);
             float tzb = t.kb == -INFINITY ? 0.f : t.zb * pow2_int(t.kb - Kb);
@@ -706,7 +728,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
         // ---- next pair ----
         g += ns;
         ++li;
-        item += n_clusters;
+        item = sh.items[li & 7];
     }
 
     // ---- release tensor memory ----
