@@ -165,13 +165,18 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Pair
     cfg.blockDim = dim3(kFinishThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = cs;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // The finish kernel may be set up while the pair kernel drains: its CTAs take the SMs the
+    // pair kernel's CTAs leave, build their tables, and wait (griddepcontrol.wait) for the pair
+    // kernel to complete before they read anything it wrote.
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, fsd_finish_kernel<DT>, fp) != cudaSuccess) return FSD_ERR_CUDA;
     return FSD_OK;
 }

@@ -247,6 +247,8 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; sh.token = -1; }
     if (tid < 64) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / 64.0));
     __syncthreads();
+    // everything above touched no global memory; what follows reads what the pair kernel wrote
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- 1. divergences, accept bits, status of this row's pairs ----
     int st = 0, first = G;
