@@ -194,6 +194,16 @@ const char *fsd_status_string(int status);
 /* Library version: major * 10000 + minor * 100 + patch. */
 int fsd_version(void);
 
+/* Measurement aid (no counterpart in the paper).  While an event is set, every verify call
+ * records it (cudaEventRecord) on the call's stream between its pair kernel and its finish
+ * kernel, so a caller that brackets the call with two events of its own can time the two
+ * kernels separately.  `event` is a cudaEvent_t passed as void*, owned by the caller; NULL
+ * clears the hook.  Process-wide and not synchronised with calls in flight on other host
+ * threads: set it, make the calls to be measured, clear it.  The record between the two
+ * kernels also keeps the finish kernel from being set up early, so timings taken with the hook
+ * are for attribution, not throughput.  Returns FSD_OK. */
+int fsd_set_stage_event(void *event);
+
 #ifdef __cplusplus
 }
 #endif

@@ -5,6 +5,7 @@ from .binding import (  # noqa: F401
     FsdError,
     fsd_default_opts,
     fsd_host_staging_bytes,
+    fsd_set_stage_event,
     fsd_status_string,
     fsd_verify_chain,
     fsd_verify_chain_host,

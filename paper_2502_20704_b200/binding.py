@@ -83,6 +83,8 @@ def _load():
         lib.fsd_status_string.argtypes = [C.c_int]
         lib.fsd_status_string.restype = C.c_char_p
         lib.fsd_version.restype = C.c_int
+        lib.fsd_set_stage_event.argtypes = [C.c_void_p]
+        lib.fsd_set_stage_event.restype = C.c_int
         _lib = lib
     return _lib
 
@@ -115,6 +117,15 @@ def fsd_status_string(status: int) -> str:
 
 def fsd_version() -> int:
     return _load().fsd_version()
+
+
+def fsd_set_stage_event(event) -> int:
+    """Record `event` (a ``torch.cuda.Event`` that has been created, a raw handle, or None) between
+    the pair kernel and the finish kernel of every later call; None clears the hook."""
+    handle = None
+    if event is not None:
+        handle = getattr(event, "cuda_event", event)
+    return _load().fsd_set_stage_event(handle)
 
 
 def fsd_workspace_bytes(B: int, positions: int, V: int, opts: FsdOpts) -> int:

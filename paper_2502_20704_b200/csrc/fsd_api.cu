@@ -3,6 +3,7 @@
 #include <climits>
 #include <cstdint>
 #include <cuda_runtime.h>
+#include <atomic>
 #include <mutex>
 
 #include "fsd_verify.h"
@@ -70,6 +71,8 @@ int finish_cluster_size(int B, int V) {
         cs <<= 1;
     return cs;
 }
+
+std::atomic<void*> g_stage_event{nullptr};   // see fsd_set_stage_event
 
 // ---- streaming kernel launch -----------------------------------------------------------
 constexpr int kMaxDev = 64;
@@ -159,6 +162,9 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Pair
         fp.records = nullptr;
     }
 
+    if (void* ev = g_stage_event.load()) {
+        if (cudaEventRecord(static_cast<cudaEvent_t>(ev), s) != cudaSuccess) return FSD_ERR_CUDA;
+    }
     const int cs = finish_cluster_size(fp.B, fp.V);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(fp.B) * cs, 1, 1);
@@ -409,5 +415,10 @@ const char* fsd_status_string(int status) {
 }
 
 int fsd_version(void) { return 100; }
+
+int fsd_set_stage_event(void* event) {
+    g_stage_event.store(event);
+    return FSD_OK;
+}
 
 }  // extern "C"
