@@ -193,6 +193,44 @@ def test_fsd_outputs_do_not_depend_on_tokens_or_accept_uniforms():
     assert np.array_equal(a.divergence, a2.divergence) and np.array_equal(a.next_token, a2.next_token)
 
 
+def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
+    """Two workloads verified at once on two streams (separate workspaces, as the header asks):
+    each must give exactly what it gives alone; a workspace reused call after call must, too."""
+    import torch
+    from paper_2502_20704_b200 import binding as fsd
+
+    ca = gi.make_chain(24, 6, 36000, dtype="bf16", recipe="zipf", sigma=(0.4, 1.2), sigma_mode="uniform", workload_id=307)
+    cb = gi.make_chain(16, 9, 52000, dtype="bf16", recipe="spike", sigma=(0.2, 2.0), sigma_mode="uniform", workload_id=308)
+    alone = [parity.run_chain_gpu(c.target, c.draft, None, None, c.u_sample, c.dtype, T=0.15) for c in (ca, cb)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    jobs = []
+    for c in (ca, cb):
+        B, g1, V = c.target.shape
+        gamma = g1 - 1
+        opts = fsd.make_opts(dtype=c.dtype, T=0.15)
+        wsb = fsd.fsd_workspace_bytes(B, gamma, V, opts)
+        jobs.append(dict(B=B, gamma=gamma, V=V, opts=opts, wsb=wsb,
+                         t=parity.to_device(c.target, c.dtype), d=parity.to_device(c.draft, c.dtype),
+                         us=parity.to_device(c.u_sample, c.dtype),
+                         acc=torch.empty(B, dtype=torch.int32, device="cuda"),
+                         tok=torch.empty(B, dtype=torch.int32, device="cuda"),
+                         D=torch.empty(B, gamma, dtype=torch.float32, device="cuda"),
+                         st=torch.empty(B, dtype=torch.int32, device="cuda"),
+                         ws=torch.full((wsb,), 0xCD, dtype=torch.uint8, device="cuda")))
+    torch.cuda.synchronize()
+    for rep in range(6):                              # interleaved: both streams always have work queued
+        for j, s in zip(jobs, streams):
+            rc = fsd.fsd_verify_chain(j["t"], j["d"], None, None, j["us"], j["B"], j["gamma"], j["V"], j["opts"],
+                                      j["acc"], j["tok"], j["D"], j["st"], j["ws"], j["wsb"], s.cuda_stream)
+            assert rc == 0, fsd.fsd_status_string(rc)
+    torch.cuda.synchronize()
+    for j, ref in zip(jobs, alone):
+        assert np.array_equal(j["acc"].cpu().numpy(), ref.accept_len)
+        assert np.array_equal(j["tok"].cpu().numpy(), ref.next_token)
+        assert np.array_equal(j["D"].cpu().numpy(), ref.divergence)
+        assert not j["st"].cpu().numpy().any()
+
+
 def test_out_of_range_draft_token_is_rejected_in_sd_mode():
     c = gi.make_chain(2, 3, 512, dtype="f32", recipe="spike", sigma=(0.1,), workload_id=305)
     c.draft_tokens[0, 1] = 512
