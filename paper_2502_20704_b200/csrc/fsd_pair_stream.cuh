@@ -508,6 +508,17 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
                         const float ca = ka == -INFINITY ? 0.f : -ka, cb = kb == -INFINITY ? 0.f : -kb;
                         ca2 = pack2(ca, ca); cb2 = pack2(cb, cb);
                     }
+                    // This warp is done with the slot: every lane's vectors are in registers (the vote
+                    // above consumed them).  Nobody waits for the slot to drain: one stage later, when
+                    // every warp has long left it, this stage's duty warp refills it.
+                    if (lane == 0) {
+                        mbar_arrive(&sh.empty[slot]);
+                        if (gs > 0 && warp == static_cast<int>(gs % kStreamWarps)) {
+                            const uint32_t ps = gs - 1;
+                            mbar_wait(&sh.empty[ps % kRing], (ps / kRing) & 1, P.timeout_flag, dead);
+                            issue_stage(ps + kRing);
+                        }
+                    }
                     float e[VPT][EPT];
 #pragma unroll
                     for (int v = 0; v < VPT; ++v) {
@@ -555,17 +566,6 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
 #pragma unroll
                                 for (int j = 0; j < EPT; ++j) ereg[(s - NT < 0 ? 0 : s - NT) * EPS + v * EPT + j] = e[v][j];
                             }
-                        }
-                    }
-                    // This warp is done with the slot.  Nobody waits for the slot to drain: one stage
-                    // later, when every warp has long left it, this stage's duty warp refills it.
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(&sh.empty[slot]);
-                        if (gs > 0 && warp == static_cast<int>(gs % kStreamWarps)) {
-                            const uint32_t ps = gs - 1;
-                            mbar_wait(&sh.empty[ps % kRing], (ps / kRing) & 1, P.timeout_flag, dead);
-                            issue_stage(ps + kRing);
                         }
                     }
                 }
