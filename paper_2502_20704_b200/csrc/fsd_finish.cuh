@@ -468,17 +468,37 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         return;
     }
 
-    // ---- CTA-local maxima (exact); for the greedy FSD choice also the argmax of the logits ----
+    // ---- references.  A residual draw follows a rejection, so the rejected pair's record has
+    //      references (log2 domain) for both rows, near their maxima and common to the cluster;
+    //      otherwise one pass for the CTA-local maxima (exact), and for the greedy FSD choice the
+    //      argmax of the logits ----
+    double kra = 0.0, krb = 0.0;
+    bool common = false;
+    if (residual0 && P.records != nullptr) {
+        const PairRecord* r = P.records + (static_cast<size_t>(b) * G + n);
+        if (r->state & kRecordStats) {
+            float fa = -INFINITY, fb = -INFINITY;
+            bool nan = false;
+            for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
+                const float a = r->part[c].ka, q = r->part[c].kb;
+                nan = nan || a != a || q != q;
+                fa = fmaxf(fa, a); fb = fmaxf(fb, q);
+            }
+            if (!nan && isfinite(fa) && isfinite(fb)) { kra = fa; krb = fb; common = true; }
+        }
+    }
     float mx[2] = {-INFINITY, -INFINITY};
     int amax = 0x7fffffff;
     float amax_v = -INFINITY;
-    for_chunk<DT>(a_row, b_row, k0, k1, vec, residual0, [&](int k, float xa, float xb) {
-        if (xa > amax_v) { amax_v = xa; amax = k; }
-        mx[1] = fmaxf(mx[1], xb);
-    });
-    mx[0] = amax_v;
-    block_max<2>(mx, sh.red_f);
-    const double Ra = mx[0], Rb = mx[1];                 // this CTA's references
+    if (!common) {
+        for_chunk<DT>(a_row, b_row, k0, k1, vec, residual0, [&](int k, float xa, float xb) {
+            if (xa > amax_v) { amax_v = xa; amax = k; }
+            mx[1] = fmaxf(mx[1], xb);
+        });
+        mx[0] = amax_v;
+        block_max<2>(mx, sh.red_f);
+    }
+    const double Ra = common ? 0.0 : mx[0], Rb = common ? 0.0 : mx[1];   // this CTA's references (logit domain)
 
     if (greedy && !residual0) {
         // argmax of P_T == argmax of the logits, ties to the lowest index
@@ -526,8 +546,13 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     if (residual0) {
         double z[2] = {0.0, 0.0};
         for_chunk<DT>(a_row, b_row, k0, k1, vec, true, [&](int, float xa, float xb) {
-            if (Ra > -INFINITY) z[0] += exp2_table((static_cast<double>(xa) - Ra) * kLog2eD, tab);
-            if (Rb > -INFINITY) z[1] += exp2_table((static_cast<double>(xb) - Rb) * kLog2eD, tab);
+            if (common) {
+                z[0] += exp2_table(fma(static_cast<double>(xa), kLog2eD, -kra), tab);
+                z[1] += exp2_table(fma(static_cast<double>(xb), kLog2eD, -krb), tab);
+            } else {
+                if (Ra > -INFINITY) z[0] += exp2_table((static_cast<double>(xa) - Ra) * kLog2eD, tab);
+                if (Rb > -INFINITY) z[1] += exp2_table((static_cast<double>(xb) - Rb) * kLog2eD, tab);
+            }
         });
         block_sum<2>(z, sh.red_d);
         mine.d[0] = Ra; mine.d[1] = Rb; mine.d[2] = z[0]; mine.d[3] = z[1]; mine.i[0] = 0; mine.i[1] = 0;
@@ -551,6 +576,12 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     for (int attempt = 0; attempt < 2; ++attempt) {
         // weight of one vocabulary entry: P_T relative to this CTA's maximum, or the SD residual
         auto weight = [&](float xa, float xb) -> double {
+            if (common) {
+                const double pa = exp2_table(fma(static_cast<double>(xa), kLog2eD, -kra), tab);
+                if (!residual) return pa;
+                const double r = pa * iZa - exp2_table(fma(static_cast<double>(xb), kLog2eD, -krb), tab) * iZb;
+                return r > 0.0 ? r : 0.0;
+            }
             if (!residual) return Ra > -INFINITY ? exp2_table((static_cast<double>(xa) - Ra) * kLog2eD, tab) : 0.0;
             const double r = exp2_table((static_cast<double>(xa) - Ma) * kLog2eD, tab) * iZa -
                              exp2_table((static_cast<double>(xb) - Mb) * kLog2eD, tab) * iZb;
@@ -562,7 +593,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             const double w = weight(xa, xb);
             csum += w;
             if (w > 0.0) lastp = k;
-            if (w > wbest) { wbest = w; kbest = k; }
+            if (greedy && w > wbest) { wbest = w; kbest = k; }
         });
         // inclusive / exclusive scan of the chunk sums over the CTA, fixed order
         double incl = csum;
@@ -656,15 +687,29 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         const int c = sh.cand;
         if (c == 0x7fffffff) {                            // crossing lost to rounding inside this CTA
             if (tid == 0) P.next_token[b] = sh.last_pos;
-        } else if (tid == c) {
-            double running = excl;
-            int tok = lastp;
-            bool found = false;
-            for_chunk<DT>(a_row, b_row, k0, k1, vec, residual, [&](int k, float xa, float xb) {
-                running += weight(xa, xb);
-                if (!found && running > t_local) { tok = k; found = true; }
-            });
-            P.next_token[b] = tok;
+        } else if (warp == (c >> 5)) {
+            // the warp of the thread whose chunk holds the crossing walks that chunk together
+            const int src = c & 31;
+            const int ck0 = __shfl_sync(0xffffffffu, k0, src), ck1 = __shfl_sync(0xffffffffu, k1, src);
+            double base = __shfl_sync(0xffffffffu, excl, src);
+            int tok = 0x7fffffff;
+            const int fallback = __shfl_sync(0xffffffffu, lastp, src);
+            for (int kb = ck0; kb < ck1; kb += 32) {
+                const int k = kb + lane;
+                double w = 0.0;
+                if (k < ck1) w = weight(load_logit<DT>(a_row, k), residual ? load_logit<DT>(b_row, k) : 0.f);
+                double run = w;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const double up = __shfl_up_sync(0xffffffffu, run, d);
+                    if (lane >= d) run += up;
+                }
+                run += base;
+                if (k < ck1 && run > t_local && k < tok) tok = k;
+                base = __shfl_sync(0xffffffffu, run, 31);
+            }
+            tok = __reduce_min_sync(0xffffffffu, tok);
+            if (lane == 0) P.next_token[b] = tok != 0x7fffffff ? tok : fallback;
         }
         return;
     }
