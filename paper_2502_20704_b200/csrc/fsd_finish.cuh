@@ -49,11 +49,13 @@ struct FinishExchange {        // what one CTA publishes to its cluster
     double d[4];
     int i[2];
 };
+constexpr int kExpTable = 256;
+
 struct FinishShared {
     FinishExchange slot;
     double gather_d[kMaxClusterSize];   // one value per CTA of the cluster (see cluster_gather)
     int gather_i[kMaxClusterSize];
-    double exp_table[64];      // 2^(j/64)
+    double exp_table[kExpTable];   // 2^(j/256)
     double red_d[32 * 2];
     float red_f[32 * 2];
     double warp_tot[32];
@@ -68,21 +70,22 @@ struct FinishShared {
     int8_t tree_bit[kMaxTreeNodes];
 };
 
-// 2^y in double precision for y <= 0 (relative error about 2e-16); 0 below the normal range.
+// 2^y in double precision (relative error about 2e-16) for -1000 < y < 1000; 0 below, NaN for NaN.
+// y = (k + r) / 256 with integer k and |r| <= 1/2: 2^y = 2^(k >> 8) * table[k & 255] * 2^(r/256),
+// the last factor by a degree-4 polynomial in r (|r ln2 / 256| <= 1.4e-3, remainder < 5e-17).
 __device__ __forceinline__ double exp2_table(double y, const double* table) {
     if (!(y > -1000.0)) return y != y ? y : 0.0;
-    const double kMagic = 6755399441055744.0;                      // 1.5 * 2^52: the sum's low word is round(64 y)
-    const double t = fma(y, 64.0, kMagic);
+    const double kMagic = 6755399441055744.0;                      // 1.5 * 2^52: the sum's low word is round(256 y)
+    const double t = fma(y, 256.0, kMagic);
     const int k = __double2loint(t);
-    const double r = fma(t - kMagic, -1.0 / 64.0, y);              // |r| <= 1/128, exact
-    const double z = r * kLn2D;
-    double p = fma(z, 1.0 / 120.0, 1.0 / 24.0);
-    p = fma(p, z, 1.0 / 6.0);
-    p = fma(p, z, 0.5);
-    p = fma(p, z, 1.0);
-    p = fma(p, z, 1.0);
-    const double m = table[k & 63] * p;                            // in [1, 2.0001)
-    const int hi = __double2hiint(m) + ((k >> 6) << 20);           // scale by 2^(k >> 6): stays normal for y > -1000
+    const double r = fma(y, 256.0, kMagic - t);                    // 256 y - k, exact: |r| <= 1/2
+    // coefficients (ln2 / 256)^i / i!
+    double p = fma(r, 2.239395190875157e-12, 3.308302680541371e-09);
+    p = fma(p, r, 3.665565596910106e-06);
+    p = fma(p, r, 2.7076061740622863e-03);
+    p = fma(p, r, 1.0);
+    const double m = table[k & (kExpTable - 1)] * p;               // in [1, 2.0001)
+    const int hi = __double2hiint(m) + ((k >> 8) << 20);           // scale by 2^(k >> 8): stays normal for |y| < 1000
     return __hiloint2double(hi, __double2loint(m));
 }
 
@@ -245,7 +248,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const bool tree = P.parent != nullptr;
 
     if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; sh.token = -1; }
-    if (tid < 64) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / 64.0));
+    if (tid < kExpTable) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / kExpTable));
     __syncthreads();
     // everything above touched no global memory; what follows reads what the pair kernel wrote
     asm volatile("griddepcontrol.wait;" ::: "memory");
