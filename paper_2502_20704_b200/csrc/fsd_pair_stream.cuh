@@ -2,10 +2,11 @@
 //
 // A (row, position) pair is split along the vocabulary over a thread-block cluster of C CTAs
 // (C = 1, 2, 4 or 8, the smallest that lets a CTA's slice fit on chip).  Clusters are
-// persistent and walk the pair list round-robin.  Per pair, each CTA
+// persistent and claim pairs from a shared counter.  Per pair, each CTA
 //   1. receives its slice of both rows in shared memory through a ring of bulk asynchronous
-//      copies (cp.async.bulk + mbarrier).  A ring slot is refilled as soon as its last reader
-//      is done, so the next pair's slices stream in while this pair is finished;
+//      copies (cp.async.bulk + mbarrier).  A warp releases a slot as soon as its vectors are in
+//      registers; the slot is refilled one stage later by a rotating duty warp, so the next
+//      pair's slices stream in while this pair is finished and nobody waits for a slot to drain;
 //   2. sweeps each stage once as it lands: e = 2^(logit * log2e - k) with one MUFU ex2 per
 //      logit, the sums Z = sum e and S = sum e*y (or the KL sum), a bitwise "rows differ" flag,
 //      and parks the e values in tensor memory (128 per thread) and registers (32).  k is a
@@ -39,7 +40,7 @@ constexpr int kVecPerThread = 2;                           // 16-byte vectors pe
 constexpr int kStageVecs = kStreamThreads * kVecPerThread; // vectors per row and stage
 constexpr int kStageRowBytes = kStageVecs * 16;
 constexpr int kStageBytes = 2 * kStageRowBytes;
-constexpr int kMaxStagesPerPair = kRing - 1;               // a pair's slice must be resident at once
+constexpr int kMaxStagesPerPair = kRing - 1;               // stages of e values a thread can park (4 in tensor memory, 1 in registers)
 constexpr int kTmemCols = 256;                             // per CTA: 8 warps -> 2 per lane quarter x 128 columns
 constexpr int kTmemPerThread = 128;
 constexpr int kMaxVecPerCta = kMaxStagesPerPair * kStageVecs;
@@ -58,7 +59,8 @@ struct alignas(16) Stats {
     float za, zb;
     float s0, sb;
     float x;                   // second-sweep sum of the PREVIOUS pair (in flight only)
-    uint32_t diff;             // 0: the two rows are bitwise identical so far
+    uint32_t diff;             // 0: the two rows are bitwise identical so far (bit 0 once a CTA has folded it;
+                               // rank 0's message carries the next claimed pair id in the bits above)
 };
 static_assert(sizeof(Stats) == 32, "Stats travels as two 16-byte stores");
 
@@ -355,9 +357,9 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     bool dead = false;                               // a bounded wait of this thread ran out
 
     // ---- producer: stage number -> (pair, slice part); any thread may issue a stage ----
-    // Stage gg of this CTA is part gg % ns of the (gg / ns)-th pair of this cluster.  The warp
-    // that is last to finish reading a ring slot refills it at once (see sweep B), so the
-    // copies are issued as early as possible and the work is spread over the warps.
+    // Stage gg of this CTA is part gg % ns of the (gg / ns)-th pair of this cluster (its id is in
+    // sh.items).  Stage gg + kRing is issued by the duty warp of stage gg + 1 (see sweep B), so the
+    // copies go out early and the work is spread over the warps.
     auto issue_stage = [&](uint32_t gg) {
         const uint32_t k = gg / static_cast<uint32_t>(ns), s = gg - k * static_cast<uint32_t>(ns);
         const int item = sh.items[k & 7];
