@@ -358,7 +358,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
 
     // ---- producer: stage number -> (pair, slice part); any thread may issue a stage ----
     // Stage gg of this CTA is part gg % ns of the (gg / ns)-th pair of this cluster (its id is in
-    // sh.items).  Stage gg + kRing is issued by the duty warp of stage gg + 1 (see sweep B), so the
+    // sh.items).  Stage gg + kRing is issued by the duty warp of stage gg + 1 (see the first sweep), so the
     // copies go out early and the work is spread over the warps.
     auto issue_stage = [&](uint32_t gg) {
         const uint32_t k = gg / static_cast<uint32_t>(ns), s = gg - k * static_cast<uint32_t>(ns);
@@ -412,7 +412,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
             bad = pr < -1 || pr >= i;
         }
 
-        // ---- sweep B: exponentials, sums, park the e values; then this warp's statistics ----
+        // ---- first sweep: exponentials, sums, park the e values; then this warp's statistics ----
         float ka = -INFINITY, kb = -INFINITY;
         Stats mine;
         mine.ka = -INFINITY; mine.kb = -INFINITY; mine.za = 0.f; mine.zb = 0.f; mine.s0 = 0.f; mine.sb = 0.f;
