@@ -1,0 +1,48 @@
+"""GPU-vs-oracle parity on seeded random shapes, dtypes, divergences, modes and thresholds.
+
+The named workloads fix a handful of shapes; this sweep draws others (vocabulary sizes that are
+and are not multiples of the vector width, cluster sizes 1 to 8, one to five ring stages per
+pair, masked entries) so that every launch configuration of the pair kernels meets the oracle.
+"""
+
+import numpy as np
+import pytest
+
+import fsd_inputs as gi
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(it: int):
+    rng = np.random.default_rng(20704 + it)
+    dtype = str(rng.choice(["bf16", "f32"]))
+    V = int(rng.choice([8 * rng.integers(8, 400), 8 * rng.integers(400, 6000), 8 * rng.integers(6000, 20000),
+                        int(rng.integers(9, 5000))]))
+    B, gamma = int(rng.integers(1, 40)), int(rng.integers(1, 12))
+    if B * gamma * V > 3e7:
+        B = max(1, int(3e7 / (gamma * V)))
+    opts = dict(div=str(rng.choice(["js", "kl", "tv"])), mode=str(rng.choice(["fsd", "fsd", "sd", "rfsd"])),
+                sample=str(rng.choice(["invcdf", "invcdf", "greedy"])), cmp=str(rng.choice(["lt", "le"])),
+                T=float(rng.choice([0.0, 0.02, 0.1, 0.3, 0.7, 2.0])))
+    recipe = str(rng.choice(["spike", "zipf"]))
+    c = gi.make_chain(B, gamma, V, dtype=dtype, recipe=recipe, sigma=(0.1, 2.0), sigma_mode="uniform",
+                      disjoint_frac=0.1 if recipe == "zipf" else 0.0, workload_id=2000 + it)
+    if rng.random() < 0.3:                          # masked vocabulary entries (same mask in every row)
+        f32 = dtype == "f32"
+        t = c.target if f32 else gi.bf16_bits_to_f32(c.target)
+        d = c.draft if f32 else gi.bf16_bits_to_f32(c.draft)
+        t[:, :, rng.random(V) < 0.3] = -np.inf
+        if rng.random() < 0.5:
+            d[:, :, rng.random(V) < 0.2] = -np.inf
+        if not f32:
+            c.target[:] = gi.f32_to_bf16_bits(t)
+            c.draft[:] = gi.f32_to_bf16_bits(d)
+    return c, opts
+
+
+@pytest.mark.parametrize("it", range(24))
+def test_random_shape_matches_oracle(it):
+    c, opts = _case(it)
+    r = parity.check_chain(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, **opts)
+    assert r["max_err"] < (1e-5 if c.dtype == "f32" else 1e-4)
