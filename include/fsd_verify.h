@@ -165,7 +165,7 @@ int fsd_verify_chain_host(const void *h_target_logits, const void *h_draft_logit
  * device budget is already handed out.  Such a caller has no buffer to pass as `workspace` and
  * cannot call cudaMalloc to get one.  This variant computes exactly what fsd_verify_chain
  * computes, with the same kernels, but keeps the per-position scratch (accept bits, status words
- * and the 304-byte record of each position) in a fixed array that is part of the library's device image, so the caller passes only inputs and
+ * and the 592-byte record of each position) in a fixed array that is part of the library's device image, so the caller passes only inputs and
  * outputs.  It calls no cudaMalloc, cudaFree or any other allocating routine.
  *
  * Limits and rules
@@ -181,7 +181,7 @@ int fsd_verify_chain_host(const void *h_target_logits, const void *h_draft_logit
  *     separate workspaces.
  * Arguments, outputs and the other error codes are those of fsd_verify_chain. */
 #define FSD_STATIC_SCRATCH_BYTES 786432
-#define FSD_STATIC_MAX_POSITIONS 2048
+#define FSD_STATIC_MAX_POSITIONS 1024
 int fsd_verify_chain_static(const void *target_logits, const void *draft_logits,
                             const int32_t *draft_tokens, const float *u_accept, const float *u_sample,
                             int B, int gamma, int V, const fsd_opts *opts,

@@ -24,7 +24,7 @@ DTYPES = {"f32": 0, "bf16": 1}
 FSD_OK = 0
 FSD_ERR_NULL, FSD_ERR_SHAPE, FSD_ERR_ALIGN, FSD_ERR_ENUM = -1, -2, -3, -4
 FSD_ERR_WORKSPACE, FSD_ERR_UNSUPPORTED, FSD_ERR_CUDA, FSD_ERR_TOO_LARGE = -5, -6, -7, -8
-FSD_STATIC_MAX_POSITIONS = 2048
+FSD_STATIC_MAX_POSITIONS = 1024
 FSD_ROW_NONFINITE, FSD_ROW_TIMEOUT, FSD_ROW_BADTREE = 1, 2, 4
 
 

@@ -128,15 +128,15 @@ struct PairTotals {
 __device__ __forceinline__ double pow2_int_d(double d) {
     return d < -1022.0 ? 0.0 : __hiloint2double((1023 + static_cast<int>(d)) << 20, 0);
 }
-__device__ __forceinline__ double group8_sum(double v) {
+__device__ __forceinline__ double group_sum(double v) {       // over the kStreamMaxCluster lanes of a record
 #pragma unroll
-    for (int m = 4; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
     return v;
 }
-// Called by all 32 lanes: lane 8*q + r folds part r of the record `rec` of group q (null: no
+// Called by all 32 lanes: lane 16*q + r folds part r of the record `rec` of group q (null: no
 // record for this group); every lane of a group returns the group's totals.
 __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
-    const int r = threadIdx.x & 7;
+    const int r = threadIdx.x & (kStreamMaxCluster - 1);
     PairTotals t;
     Stats c;
     c.ka = -INFINITY; c.kb = -INFINITY; c.za = 0.f; c.zb = 0.f; c.s0 = 0.f; c.sb = 0.f; c.x = 0.f; c.diff = 0;
@@ -144,7 +144,7 @@ __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     if (rec != nullptr && r < static_cast<int>(rec->ncta)) { c = rec->part[r]; x = rec->x[r]; }
     float ka = c.ka, kb = c.kb;                          // NaN references win
 #pragma unroll
-    for (int m = 4; m > 0; m >>= 1) {
+    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) {
         const float oa = __shfl_xor_sync(0xffffffffu, ka, m), ob = __shfl_xor_sync(0xffffffffu, kb, m);
         ka = (oa != oa || ka != ka) ? __int_as_float(0x7fc00000) : fmaxf(ka, oa);
         kb = (ob != ob || kb != kb) ? __int_as_float(0x7fc00000) : fmaxf(kb, ob);
@@ -154,22 +154,22 @@ __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     const double db = c.kb == -INFINITY ? 0.0 : static_cast<double>(c.kb) - kb;
     const double fa = (c.ka == -INFINITY || da != da) ? 0.0 : pow2_int_d(da);
     const double fb = (c.kb == -INFINITY || db != db) ? 0.0 : pow2_int_d(db);
-    t.Za = group8_sum(fa * c.za); t.Zb = group8_sum(fb * c.zb);
+    t.Za = group_sum(fa * c.za); t.Zb = group_sum(fb * c.zb);
     t.Sa = 0.0; t.Sb = 0.0; t.K = 0.0;
     if (div == FSD_DIV_KL) {
         const bool inf = c.s0 == INFINITY;
         const double k = inf ? 0.0 : fa * (static_cast<double>(c.s0) + (da - db) * c.za);
-        t.K = group8_sum(k);
-        const unsigned any_inf = __ballot_sync(0xffffffffu, inf) >> (threadIdx.x & 24) & 0xffu;
+        t.K = group_sum(k);
+        const unsigned any_inf = __ballot_sync(0xffffffffu, inf) >> (threadIdx.x & 16) & 0xffffu;
         if (any_inf) t.K = static_cast<double>(INFINITY);
     } else {
-        t.Sa = group8_sum(fa * (static_cast<double>(c.s0) + da * c.za));
-        t.Sb = group8_sum(fb * (static_cast<double>(c.sb) + db * c.zb));
+        t.Sa = group_sum(fa * (static_cast<double>(c.s0) + da * c.za));
+        t.Sb = group_sum(fb * (static_cast<double>(c.sb) + db * c.zb));
     }
-    t.X = group8_sum(static_cast<double>(x));
+    t.X = group_sum(static_cast<double>(x));
     uint32_t df = c.diff;
 #pragma unroll
-    for (int m = 4; m > 0; m >>= 1) df |= __shfl_xor_sync(0xffffffffu, df, m);
+    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) df |= __shfl_xor_sync(0xffffffffu, df, m);
     t.differ = df;
     return t;
 }
@@ -256,12 +256,12 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     // ---- 1. divergences, accept bits, status of this row's pairs ----
     int st = 0, first = G;
     if (P.records != nullptr) {
-        // four pairs per warp: eight lanes fold a pair's record, the first of them judges it
-        for (int i0 = 4 * warp; i0 < G; i0 += 4 * (blockDim.x >> 5)) {
-            const int i = i0 + (lane >> 3);
+        // two pairs per warp: sixteen lanes fold a pair's record, the first of them judges it
+        for (int i0 = 2 * warp; i0 < G; i0 += 2 * (blockDim.x >> 5)) {
+            const int i = i0 + (lane >> 4);
             const int item = b * G + i;
             const PairTotals tot = fold_record(i < G ? P.records + item : nullptr, P.div);
-            if (i < G && (lane & 7) == 0) {
+            if (i < G && (lane & 15) == 0) {
                 int trow = i;
                 if (tree) {
                     const int par = P.parent[item];

@@ -1,7 +1,7 @@
 // Streaming per-(row, position) kernel: every logit is read from HBM once.
 //
 // A (row, position) pair is split along the vocabulary over a thread-block cluster of C CTAs
-// (C = 1, 2, 4 or 8, the smallest that lets a CTA's slice fit on chip).  Clusters are
+// (C = 1, 2, 4, 8 or 16, the smallest that lets a CTA's slice fit on chip).  Clusters are
 // persistent and claim pairs from a shared counter.  Per pair, each CTA
 //   1. receives its slice of both rows in shared memory through a ring of bulk asynchronous
 //      copies (cp.async.bulk + mbarrier).  A warp releases a slot as soon as its vectors are in
@@ -45,7 +45,7 @@ constexpr int kTmemCols = 256;                             // per CTA: 8 warps -
 constexpr int kTmemPerThread = 128;
 constexpr int kMaxVecPerCta = kMaxStagesPerPair * kStageVecs;
 constexpr int kMaxClusterSize = 8;                        // finish kernel (portable size)
-constexpr int kStreamMaxCluster = 8;                       // streaming kernel
+constexpr int kStreamMaxCluster = 16;                      // streaming kernel (above 8: the non-portable opt-in)
 constexpr int kStreamCtasPerSm = 2;
 constexpr uint32_t kSpinLimit = 1u << 24;                  // polls before a wait gives up
 
@@ -73,7 +73,7 @@ struct alignas(16) PairRecord {
     uint32_t state;            // kRecordStats | kRecordBadTree
     uint32_t pad[2];
 };
-static_assert(sizeof(PairRecord) == 304, "PairRecord layout");
+static_assert(sizeof(PairRecord) == 592, "PairRecord layout");
 constexpr uint32_t kRecordStats = 1, kRecordBadTree = 2;
 
 struct StreamParams {

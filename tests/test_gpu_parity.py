@@ -193,6 +193,17 @@ def test_fsd_outputs_do_not_depend_on_tokens_or_accept_uniforms():
     assert np.array_equal(a.divergence, a2.divergence) and np.array_equal(a.next_token, a2.next_token)
 
 
+@pytest.mark.parametrize("dtype,V", [("f32", 100000), ("f32", 152064), ("bf16", 200008), ("bf16", 256000)])
+def test_vocabularies_that_need_sixteen_cta_clusters(dtype, V):
+    """Rows too long for eight CTAs' on-chip capacity (fp32 above 81920 entries, bf16 above
+    163840) are streamed by clusters of sixteen."""
+    c = gi.make_chain(5, 4, V, dtype=dtype, recipe="zipf", sigma=(0.3, 1.5), sigma_mode="uniform",
+                      disjoint_frac=0.1, workload_id=309)
+    for div in ("js", "kl", "tv"):
+        _check(c, div=div, T=0.25)
+    _check(c, mode="rfsd", T=0.25)
+
+
 def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
     """Two workloads verified at once on two streams (separate workspaces, as the header asks):
     each must give exactly what it gives alone; a workspace reused call after call must, too."""
