@@ -204,6 +204,42 @@ int fsd_version(void);
  * are for attribution, not throughput.  Returns FSD_OK. */
 int fsd_set_stage_event(void *event);
 
+/* ---- Threshold tuning (Section "Selecting T"; Discussion, "Potential further developments") ----
+ * The paper tunes T on a small development set by running FSD at candidate thresholds and
+ * looking at the speed each gives, and notes that FSD's decisions are a deterministic function
+ * of the two distributions.  Everything such a sweep needs is in the divergences a verify call
+ * returns, so these three helpers work on `divergence` ([B, positions] float, device, row-major,
+ * as written by fsd_verify_chain; values >= 0, +inf, or NaN for non-finite inputs) and never touch
+ * logits.  The accepted length of a row at threshold T is the index of its first position that
+ * fails `D compare T` (NaN never passes); the speed proxy is its mean over the rows.  All pointers
+ * are device pointers owned by the caller; the calls are asynchronous on `stream`, allocate
+ * nothing and need no workspace.  Errors: FSD_ERR_NULL, FSD_ERR_SHAPE (B < 1, positions < 1,
+ * n_thresholds < 1, target negative or NaN), FSD_ERR_ENUM (compare), FSD_ERR_CUDA. */
+
+/* For each of `n_thresholds` candidate thresholds (device array): the mean accepted length over
+ * the B rows and the accepted fraction of all B * positions positions. */
+int fsd_threshold_sweep(const float *divergence, int B, int positions,
+                        const float *thresholds, int n_thresholds, int compare,
+                        float *mean_accept_len,   /* [n_thresholds] out */
+                        float *accept_fraction,   /* [n_thresholds] out */
+                        void *stream);
+
+/* The smallest float T >= 0 whose mean accepted length is at least `target_mean_accept_len`
+ * (ceil(target * B) positions accepted, at most B * positions), and the mean it achieves.  +inf if
+ * no finite threshold gets there (rows cut short by NaN, or by +inf under FSD_CMP_LT). */
+int fsd_calibrate_threshold(const float *divergence, int B, int positions,
+                            float target_mean_accept_len, int compare,
+                            float *threshold_out,  /* [1] out */
+                            float *achieved_out,   /* [1] out: mean accepted length at threshold_out */
+                            void *stream);
+
+/* labels[b, i] = 1 if position (b, i) alone passes `D compare threshold`, else 0 (NaN: 0): the
+ * token-level accept / reject labels the paper's Discussion proposes to learn from; the prefix
+ * rule is not applied. */
+int fsd_accept_labels(const float *divergence, int B, int positions, float threshold, int compare,
+                      uint8_t *labels,             /* [B, positions] out */
+                      void *stream);
+
 #ifdef __cplusplus
 }
 #endif

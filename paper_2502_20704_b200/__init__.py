@@ -3,10 +3,13 @@
 from .binding import (  # noqa: F401
     FsdOpts,
     FsdError,
+    fsd_accept_labels,
+    fsd_calibrate_threshold,
     fsd_default_opts,
     fsd_host_staging_bytes,
     fsd_set_stage_event,
     fsd_status_string,
+    fsd_threshold_sweep,
     fsd_verify_chain,
     fsd_verify_chain_host,
     fsd_verify_chain_static,

@@ -85,6 +85,12 @@ def _load():
         lib.fsd_version.restype = C.c_int
         lib.fsd_set_stage_event.argtypes = [C.c_void_p]
         lib.fsd_set_stage_event.restype = C.c_int
+        lib.fsd_threshold_sweep.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, C.c_int, vp, vp, C.c_void_p]
+        lib.fsd_threshold_sweep.restype = C.c_int
+        lib.fsd_calibrate_threshold.argtypes = [vp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, C.c_void_p]
+        lib.fsd_calibrate_threshold.restype = C.c_int
+        lib.fsd_accept_labels.argtypes = [vp, C.c_int, C.c_int, C.c_float, C.c_int, vp, C.c_void_p]
+        lib.fsd_accept_labels.restype = C.c_int
         _lib = lib
     return _lib
 
@@ -182,3 +188,20 @@ def fsd_verify_chain_static(target_logits, draft_logits, draft_tokens, u_accept,
                                            _ptr(u_accept), _ptr(u_sample), B, gamma, V,
                                            C.byref(opts) if opts is not None else None, _ptr(accept_len),
                                            _ptr(next_token), _ptr(divergence), _ptr(row_status), _ptr(stream))
+
+
+
+def fsd_threshold_sweep(divergence, B, positions, thresholds, n_thresholds, compare, mean_accept_len,
+                        accept_fraction, stream=None) -> int:
+    return _load().fsd_threshold_sweep(_ptr(divergence), B, positions, _ptr(thresholds), n_thresholds, compare,
+                                       _ptr(mean_accept_len), _ptr(accept_fraction), stream)
+
+
+def fsd_calibrate_threshold(divergence, B, positions, target_mean_accept_len, compare, threshold_out, achieved_out,
+                            stream=None) -> int:
+    return _load().fsd_calibrate_threshold(_ptr(divergence), B, positions, float(target_mean_accept_len), compare,
+                                           _ptr(threshold_out), _ptr(achieved_out), stream)
+
+
+def fsd_accept_labels(divergence, B, positions, threshold, compare, labels, stream=None) -> int:
+    return _load().fsd_accept_labels(_ptr(divergence), B, positions, float(threshold), compare, _ptr(labels), stream)

@@ -11,6 +11,7 @@
 #include "fsd_finish.cuh"
 #include "fsd_pair_generic.cuh"
 #include "fsd_pair_stream.cuh"
+#include "fsd_tuning.cuh"
 
 namespace {
 
@@ -419,6 +420,38 @@ int fsd_version(void) { return 100; }
 int fsd_set_stage_event(void* event) {
     g_stage_event.store(event);
     return FSD_OK;
+}
+
+int fsd_threshold_sweep(const float* divergence, int B, int positions, const float* thresholds, int n_thresholds,
+                        int compare, float* mean_accept_len, float* accept_fraction, void* stream) {
+    if (divergence == nullptr || thresholds == nullptr || mean_accept_len == nullptr || accept_fraction == nullptr)
+        return FSD_ERR_NULL;
+    if (B < 1 || positions < 1 || n_thresholds < 1) return FSD_ERR_SHAPE;
+    if (compare != FSD_CMP_LT && compare != FSD_CMP_LE) return FSD_ERR_ENUM;
+    fsd_threshold_sweep_kernel<<<n_thresholds, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        divergence, B, positions, thresholds, compare, mean_accept_len, accept_fraction);
+    return cudaGetLastError() == cudaSuccess ? FSD_OK : FSD_ERR_CUDA;
+}
+
+int fsd_calibrate_threshold(const float* divergence, int B, int positions, float target_mean_accept_len, int compare,
+                            float* threshold_out, float* achieved_out, void* stream) {
+    if (divergence == nullptr || threshold_out == nullptr || achieved_out == nullptr) return FSD_ERR_NULL;
+    if (B < 1 || positions < 1 || !(target_mean_accept_len >= 0.f)) return FSD_ERR_SHAPE;   // NaN target included
+    if (compare != FSD_CMP_LT && compare != FSD_CMP_LE) return FSD_ERR_ENUM;
+    fsd_calibrate_kernel<<<1, kTuneThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        divergence, B, positions, target_mean_accept_len, compare, threshold_out, achieved_out);
+    return cudaGetLastError() == cudaSuccess ? FSD_OK : FSD_ERR_CUDA;
+}
+
+int fsd_accept_labels(const float* divergence, int B, int positions, float threshold, int compare, uint8_t* labels,
+                      void* stream) {
+    if (divergence == nullptr || labels == nullptr) return FSD_ERR_NULL;
+    if (B < 1 || positions < 1) return FSD_ERR_SHAPE;
+    if (compare != FSD_CMP_LT && compare != FSD_CMP_LE) return FSD_ERR_ENUM;
+    const size_t n = static_cast<size_t>(B) * positions;
+    const unsigned blocks = static_cast<unsigned>(n / 256 + 1 < 1184 ? n / 256 + 1 : 1184);
+    fsd_accept_labels_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(divergence, n, threshold, compare, labels);
+    return cudaGetLastError() == cudaSuccess ? FSD_OK : FSD_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -104,3 +104,15 @@ def test_status_strings():
         assert fsd.fsd_status_string(code).startswith("FSD_ERR_")
     assert "unknown" in fsd.fsd_status_string(-99)
     assert fsd.fsd_version() >= 100
+
+
+def test_tuning_entry_points_check_their_arguments_on_the_host():
+    # bad arguments are refused before anything is launched (no GPU needed)
+    assert fsd.fsd_threshold_sweep(None, 1, 1, None, 1, 0, None, None) == -1           # FSD_ERR_NULL
+    assert fsd.fsd_threshold_sweep(16, 0, 1, 16, 1, 0, 16, 16) == -2                   # FSD_ERR_SHAPE
+    assert fsd.fsd_threshold_sweep(16, 1, 1, 16, 1, 5, 16, 16) == -4                   # FSD_ERR_ENUM
+    assert fsd.fsd_calibrate_threshold(16, 1, 1, -1.0, 0, 16, 16) == -2
+    assert fsd.fsd_calibrate_threshold(16, 1, 1, float("nan"), 0, 16, 16) == -2
+    assert fsd.fsd_calibrate_threshold(None, 1, 1, 1.0, 0, 16, 16) == -1
+    assert fsd.fsd_accept_labels(16, 1, 0, 0.1, 1, 16) == -2
+    assert fsd.fsd_accept_labels(16, 1, 1, 0.1, 2, 16) == -4
