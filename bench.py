@@ -156,7 +156,7 @@ def run_reference(args, rank: int, world: int):
         "impl": "reference", "metric": "verified draft positions/sec", "value": value, "unit": "positions/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(c, rows),
+        "config": workload_config(c, rows, sampled=True),
         "cpu_baseline": {"value": value, "unit": "positions/s", "cores": orc.max_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": "positions/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -165,11 +165,15 @@ def run_reference(args, rank: int, world: int):
     print(json.dumps(line))
 
 
-def workload_config(c, B):
-    return {"workload": f"chain FSD verify B={B} gamma={c.gamma} V={c.V} {c.dtype} JS T=0.2 (config 4)",
+def workload_config(c, B, sampled=False):
+    spec = gi.CONFIGS[WORKLOAD].params
+    same = (B if not sampled else spec["B"], c.gamma, c.V, c.dtype) == (spec["B"], spec["gamma"], spec["V"], spec["dtype"])
+    mb = c.elem_size * B * (2 * c.gamma + 1) * c.V / 1e6
+    return {"workload": f"chain FSD verify B={B} gamma={c.gamma} V={c.V} {c.dtype} JS T=0.2 "
+                        + ("(config 4)" if same else "(config 4's recipe, other shape)"),
             "B": B, "gamma": c.gamma, "V": c.V, "divergence": "js", "mode": "fsd", "threshold": 0.2,
             "parallelism": "independent replicas",
-            "l2": "inputs (331 MB) exceed L2 (126 MB); 3 input copies rotated between steps"}
+            "l2": f"inputs ({mb:.0f} MB) exceed L2 (126 MB); 3 input copies rotated between steps"}
 
 
 def main():
@@ -181,6 +185,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--copies", type=int, default=3)
     ap.add_argument("--ref-rows", type=int, default=16, help="batch rows per step of the reference arm")
+    # extra rows (not the headline): the headline recipe with another vocabulary, length, batch or dtype
+    ap.add_argument("--V", type=int, default=None, help="vocabulary size instead of 152064 (e.g. 256000)")
+    ap.add_argument("--gamma", type=int, default=None, help="candidate length instead of 8 (e.g. 10, 15, 20)")
+    ap.add_argument("--B", type=int, default=None, help="batch rows instead of 64")
+    ap.add_argument("--dtype", default=None, choices=["bf16", "f32"], help="logit type instead of bf16")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -223,12 +232,19 @@ def main():
         return float(t.item())
 
     # ---- workload (same seeded inputs on every rank: replicas) ----
-    c = gi.make_config(WORKLOAD)
+    overrides = {k: v for k, v in (("V", args.V), ("gamma", args.gamma), ("B", args.B), ("dtype", args.dtype))
+                 if v is not None}
+    headline = not overrides
+    c = gi.make_config(WORKLOAD, **overrides)
     T = float(gi.CONFIGS[WORKLOAD].thresholds[0])
     B, gamma, V = c.B, c.gamma, c.V
     opts = fsd.make_opts(div="js", mode="fsd", cmp="lt", sample="invcdf", dtype=c.dtype, T=T)
-    h_target = torch.from_numpy(c.target.view(np.int16)).view(torch.bfloat16).pin_memory()
-    h_draft = torch.from_numpy(c.draft.view(np.int16)).view(torch.bfloat16).pin_memory()
+    if c.dtype == "bf16":
+        h_target = torch.from_numpy(c.target.view(np.int16)).view(torch.bfloat16).pin_memory()
+        h_draft = torch.from_numpy(c.draft.view(np.int16)).view(torch.bfloat16).pin_memory()
+    else:
+        h_target = torch.from_numpy(c.target).pin_memory()
+        h_draft = torch.from_numpy(c.draft).pin_memory()
     h_us = torch.from_numpy(c.u_sample).pin_memory()
     copies = [(h_target.cuda(), h_draft.cuda()) for _ in range(max(args.copies, 1))]
     us = h_us.cuda()
@@ -305,7 +321,7 @@ def main():
     barrier()
     e2e_value, e2e_ms = aggregate_over_ranks(e0.elapsed_time(e1), float(B * gamma * args.e2e_steps), world,
                                              reduce_max, reduce_sum)
-    h2d = h_target.numel() * 2 + h_draft.numel() * 2 + h_us.numel() * 4
+    h2d = (h_target.numel() + h_draft.numel()) * c.elem_size + h_us.numel() * 4
     d2h = (h_acc.numel() + h_tok.numel() + h_D.numel() + h_st.numel()) * 4
     assert np.array_equal(h_acc.numpy(), res_acc)
 
@@ -322,9 +338,10 @@ def main():
     achieved = pair_bytes / (pair_ms * 1e-3) / 1e9
     call_achieved = ideal / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": PAIR_KERNEL_DRAM_BYTES, "peak_kind": f"of {peak_kind}",
+                "traffic": PAIR_KERNEL_DRAM_BYTES if headline else None, "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                "kernel": "fsd_pair_stream_kernel<bf16, JS> (includes the 256-byte flag memset in front of it)",
+                "kernel": "pair kernel (fsd_pair_stream_kernel<bf16, JS> on the headline workload; includes the "
+                          "256-byte flag memset in front of it)",
                 "algorithmic_bytes_per_launch": pair_bytes, "ms_per_launch": pair_ms,
                 "finish_kernel_ms": finish_ms,
                 "whole_call": {"achieved": call_achieved, "frac": call_achieved / peak,
