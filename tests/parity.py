@@ -155,3 +155,32 @@ def check_chain(inp_target, inp_draft, tokens, u_accept, u_sample, dtype, div="j
             sample_band += 1
     return dict(rows=B, band_rows=band_rows, replayed=replayed, sample_band=sample_band, max_err=max_err,
                 accept_len=g.accept_len.copy(), gpu=g, oracle=o)
+
+
+def check_tree(c, T, div="js", cmp="lt", sample="invcdf"):
+    """GPU tree verification against the oracle: divergences within tolerance; accepted depth, path
+    and token identical, with the oracle re-run on the GPU's decisions where a divergence lies
+    within D_BAND of the threshold."""
+    tol = 1e-5 if c.dtype == "f32" else 1e-4
+    g = run_tree_gpu(c.target, c.draft, c.parent, c.u_sample, c.max_depth, c.dtype, div=div, cmp=cmp, sample=sample, T=T)
+    o = orc.verify_tree(c.target, c.draft, c.parent, c.u_sample, c.max_depth, dtype=c.dtype, div=div, cmp=cmp,
+                        sample_kind=sample, T=T, band=SAMPLE_BAND)
+    compare_divergence(g.divergence, o.divergence, tol)
+    Tf = np.float32(T)
+    with np.errstate(invalid="ignore"):
+        in_band = np.abs(o.divergence - float(Tf)) < D_BAND
+    for b in range(c.B):
+        if in_band[b].any():
+            forced = np.full((1, c.N), -1, dtype=np.int8)
+            gd = g.divergence[b, in_band[b]]
+            forced[0, in_band[b]] = ((gd <= Tf) if cmp == "le" else (gd < Tf)).astype(np.int8)
+            ob = orc.verify_tree(c.target[b:b + 1], c.draft[b:b + 1], c.parent[b:b + 1], c.u_sample[b:b + 1],
+                                 c.max_depth, dtype=c.dtype, div=div, cmp=cmp, sample_kind=sample, T=T,
+                                 band=SAMPLE_BAND, forced=forced)
+            n_o, p_o, t_o, lo, hi = ob.accept_len[0], ob.path[0], ob.next_token[0], ob.tok_lo[0], ob.tok_hi[0]
+        else:
+            n_o, p_o, t_o, lo, hi = o.accept_len[b], o.path[b], o.next_token[b], o.tok_lo[b], o.tok_hi[b]
+        assert g.accept_len[b] == n_o and np.array_equal(g.path[b], p_o), f"row {b}"
+        assert g.next_token[b] == t_o or lo <= g.next_token[b] <= hi, f"row {b}: token {g.next_token[b]} vs {t_o}"
+    assert np.array_equal(g.row_status, o.row_status)
+    return g, o

@@ -63,24 +63,8 @@ def test_config4_headline_shape():
 
 def test_config5_tree():
     c = gi.make_config("c5")
-    tol = 1e-4
     for T in gi.CONFIGS["c5"].thresholds:
-        g = parity.run_tree_gpu(c.target, c.draft, c.parent, c.u_sample, c.max_depth, c.dtype, T=T)
-        o = orc.verify_tree(c.target, c.draft, c.parent, c.u_sample, c.max_depth, dtype=c.dtype, T=T,
-                            band=parity.SAMPLE_BAND)
-        parity.compare_divergence(g.divergence, o.divergence, tol)
-        in_band = np.abs(o.divergence - float(np.float32(T))) < parity.D_BAND
-        for b in range(c.B):
-            if in_band[b].any():
-                forced = np.full((1, c.N), -1, dtype=np.int8)
-                forced[0, in_band[b]] = (g.divergence[b, in_band[b]] < np.float32(T)).astype(np.int8)
-                ob = orc.verify_tree(c.target[b:b + 1], c.draft[b:b + 1], c.parent[b:b + 1], c.u_sample[b:b + 1],
-                                     c.max_depth, dtype=c.dtype, T=T, band=parity.SAMPLE_BAND, forced=forced)
-                n_o, p_o, t_o = ob.accept_len[0], ob.path[0], ob.next_token[0]
-            else:
-                n_o, p_o, t_o = o.accept_len[b], o.path[b], o.next_token[b]
-            assert g.accept_len[b] == n_o and np.array_equal(g.path[b], p_o) and g.next_token[b] == t_o
-        assert np.array_equal(g.row_status, o.row_status)
+        parity.check_tree(c, T=T)
 
 
 # --------------------------------------------------------------------------- #

@@ -46,3 +46,19 @@ def test_random_shape_matches_oracle(it):
     c, opts = _case(it)
     r = parity.check_chain(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, **opts)
     assert r["max_err"] < (1e-5 if c.dtype == "f32" else 1e-4)
+
+
+@pytest.mark.parametrize("it", range(8))
+def test_random_tree_matches_oracle(it):
+    rng = np.random.default_rng(40704 + it)
+    dtype = str(rng.choice(["bf16", "f32"]))
+    V = int(rng.choice([8 * rng.integers(16, 600), 8 * rng.integers(600, 9000), int(rng.integers(9, 3000))]))
+    B, N = int(rng.integers(1, 9)), int(rng.integers(1, 40))
+    depth, children = int(rng.integers(1, 8)), int(rng.integers(1, 5))
+    N = min(N, sum(children ** d for d in range(1, depth + 1)))      # what the limits can hold
+    if B * N * V > 2e7:
+        B = max(1, int(2e7 / (N * V)))
+    t = gi.make_tree(B, N, V, dtype=dtype, recipe=str(rng.choice(["spike", "zipf"])), sigma=float(rng.uniform(0.2, 1.5)),
+                     max_depth=depth, max_children=children, workload_id=3000 + it)
+    parity.check_tree(t, T=float(rng.choice([0.02, 0.1, 0.3, 0.7])), div=str(rng.choice(["js", "kl", "tv"])),
+                      cmp=str(rng.choice(["lt", "le"])), sample=str(rng.choice(["invcdf", "greedy"])))
