@@ -477,3 +477,91 @@ def test_nonfinite_position_is_rejected_and_flagged():
     assert np.isnan(r.divergence[1, 1])
     p, _ = orc.softmax(target[1, 1])
     assert r.next_token[1] == orc.sample(p, float(us[1]))[0]
+
+
+# --------------------------------------------------------------------------- #
+# edge rules of the token draw and of the ratio test, each worked by hand
+# --------------------------------------------------------------------------- #
+def test_residual_without_mass_falls_back_to_the_target_distribution():
+    """Eq. 3 with P_T == P_D: max(0, P_T - P_D) has no mass, so the replacement comes from P_T.
+    The rejection is forced by a draft token outside the vocabulary.  P_T = (1/2,1/4,1/8,1/8):
+    CDF (.5,.75,.875,1) -> u = .6 gives token 1, u = .8 gives token 2, u = .9 gives token 3."""
+    p = [0.5, 0.25, 0.125, 0.125]
+    target = np.stack([_logits_of(p), _logits_of([0.25] * 4)])[None]
+    draft = _logits_of(p)[None, None]
+    toks = np.array([[4]], dtype=np.int32)
+    ua = np.zeros((1, 1), dtype=np.float32)
+    for u, want in ((0.6, 1), (0.8, 2), (0.9, 3), (0.0, 0)):
+        for mode in ("sd", "rfsd"):
+            r = orc.verify_chain(target, draft, toks, ua, np.array([u], np.float32), dtype="f32", mode=mode,
+                                 T=0.0, cmp="lt")
+            assert r.accept_len[0] == 0 and r.next_token[0] == want and r.row_status[0] == 0
+    r = orc.verify_chain(target, draft, toks, ua, np.array([0.9], np.float32), dtype="f32", mode="sd",
+                         sample_kind="greedy")
+    assert r.next_token[0] == 0                                   # argmax of P_T, not of an empty residual
+
+
+def test_rejection_on_a_nonfinite_draft_row_draws_from_the_target_distribution():
+    """SD mode, draft row with a NaN: the position is rejected and flagged, and since no residual
+    can be formed the token comes from P_T = (1/8,1/8,1/4,1/2): CDF (.125,.25,.5,1)."""
+    p = [0.125, 0.125, 0.25, 0.5]
+    target = np.stack([_logits_of(p), _logits_of([0.25] * 4)])[None]
+    draft = _logits_of([0.7, 0.1, 0.1, 0.1])[None, None].copy()
+    draft[0, 0, 1] = np.nan
+    toks = np.array([[3]], dtype=np.int32)
+    ua = np.zeros((1, 1), dtype=np.float32)
+    for u, want in ((0.05, 0), (0.2, 1), (0.3, 2), (0.7, 3)):
+        for mode in ("sd", "rfsd"):
+            r = orc.verify_chain(target, draft, toks, ua, np.array([u], np.float32), dtype="f32", mode=mode, T=5.0)
+            assert r.accept_len[0] == 0 and r.row_status[0] == orc.ST_NONFINITE
+            assert r.next_token[0] == want
+    # the same with the draft row +inf at the would-be residual's favourite token
+    draft[0, 0, 1] = np.inf
+    r = orc.verify_chain(target, draft, toks, ua, np.array([0.3], np.float32), dtype="f32", mode="sd")
+    assert r.accept_len[0] == 0 and r.next_token[0] == 2 and r.row_status[0] == orc.ST_NONFINITE
+
+
+def test_token_ids_outside_the_vocabulary_fail_the_ratio_test():
+    """Eq. 1-2 need P(x) of a token of the vocabulary: ids -1 and V never pass the ratio test,
+    whatever the uniform; under Eq. 6 such a position passes only through Div < T.
+    Position rows: p = (.1,.2,.3,.4), q = (.4,.3,.2,.1) -> JS = 0.10644 (golden case C)."""
+    p, q = [0.1, 0.2, 0.3, 0.4], [0.4, 0.3, 0.2, 0.1]
+    V = 4
+    target = np.stack([_logits_of(p)] * 3)[None].repeat(3, axis=0)          # [3, 3, V]
+    draft = np.stack([_logits_of(q)] * 2)[None].repeat(3, axis=0)           # [3, 2, V]
+    toks = np.array([[-1, 3], [3, V], [3, 3]], dtype=np.int32)              # token 3: ratio .4/.1 -> P_accept = 1
+    ua = np.zeros((3, 2), dtype=np.float32)                                 # u = 0: every in-range token passes
+    us = np.full(3, 0.5, dtype=np.float32)
+    r = orc.verify_chain(target, draft, toks, ua, us, dtype="f32", mode="sd")
+    assert r.accept_len.tolist() == [0, 1, 2]
+    assert r.accept_bits.tolist() == [[0, 1], [1, 0], [1, 1]]
+    assert np.isnan(r.p_accept[0, 0]) and np.isnan(r.p_accept[1, 1])
+    # rFSD below the divergence: the same; above it: the divergence rule accepts them
+    r = orc.verify_chain(target, draft, toks, ua, us, dtype="f32", mode="rfsd", T=0.1)
+    assert r.accept_len.tolist() == [0, 1, 2]
+    r = orc.verify_chain(target, draft, toks, ua, us, dtype="f32", mode="rfsd", T=0.11)
+    assert r.accept_len.tolist() == [2, 2, 2]
+    # a rejected out-of-range token is replaced from the residual max(0, p - q) = (0,0,.1,.3)/.4:
+    # t = .5 * .4 = .2 > .1 -> token 3
+    r = orc.verify_chain(target, draft, toks, ua, us, dtype="f32", mode="sd")
+    assert r.next_token[0] == 3 and r.next_token[1] == 3
+
+
+def test_inverse_cdf_without_a_crossing_takes_the_last_token_that_has_weight():
+    """u * W at or above the last cumulative sum (u = 1, or rounding): the largest k with
+    w_k > 0, not the last index."""
+    w = [0.25, 0.5, 0.25, 0.0, 0.0]
+    assert orc.sample(w, 1.0)[0] == 2
+    assert orc.sample(w, float(np.nextafter(np.float32(1), np.float32(0))))[0] == 2
+    assert orc.sample([0.0, 3.0, 0.0], 1.0)[0] == 1
+    assert orc.sample([0.0, 3.0, 0.0], 0.0)[0] == 1               # zero-weight entries are never chosen
+    # band edges past the total mass clamp to the same rule
+    tok, lo, hi, _ = orc.sample(w, 1.0 - 1e-9, band=1e-6)
+    assert (tok, lo, hi) == (2, 2, 2)
+    # through the chain call: a target row whose trailing entries are masked, u as close to 1 as fp32 allows
+    a = _logits_of([0.25, 0.5, 0.25, 0.0, 0.0])
+    target = np.stack([a, a])[None]
+    draft = _logits_of([0.2] * 5)[None, None]
+    us = np.array([np.nextafter(np.float32(1), np.float32(0))], dtype=np.float32)
+    r = orc.verify_chain(target, draft, None, None, us, dtype="f32", T=0.0, cmp="lt")
+    assert r.accept_len[0] == 0 and r.next_token[0] == 2
