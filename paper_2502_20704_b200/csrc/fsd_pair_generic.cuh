@@ -55,15 +55,15 @@ __device__ inline double log_prob(float logit, float M, float c, double Z) {
 }
 
 // Acceptance bit of one pair from its divergence and (for SD / rFSD) the ratio test.
-__device__ inline int accept_bit(const PairParams& P, int item, bool finite, float D,
-                                 const void* a_row, const void* b_row, int dt,
+__device__ inline int accept_bit(int mode, int cmp, float T, const int32_t* tokens, const float* u_accept, int V,
+                                 int item, bool finite, float D, const void* a_row, const void* b_row, int dt,
                                  float Ma, float ca, double Za, float Mb, float cb, double Zb) {
-    bool div_ok = finite && passes(D, P.T, P.cmp);
-    if (P.mode == FSD_MODE_FSD) return div_ok;
+    bool div_ok = finite && passes(D, T, cmp);
+    if (mode == FSD_MODE_FSD) return div_ok;
     bool ratio_ok = false;
     if (finite) {
-        const int x = P.tokens[item];
-        if (x >= 0 && x < P.V) {
+        const int x = tokens[item];
+        if (x >= 0 && x < V) {
             const float ax = dt == FSD_BF16 ? load_logit<FSD_BF16>(a_row, x) : load_logit<FSD_F32>(a_row, x);
             const float bx = dt == FSD_BF16 ? load_logit<FSD_BF16>(b_row, x) : load_logit<FSD_F32>(b_row, x);
             double pacc;                                                    // Eq. 1
@@ -73,38 +73,27 @@ __device__ inline int accept_bit(const PairParams& P, int item, bool finite, flo
                 pacc = exp(log_prob(ax, Ma, ca, Za) - log_prob(bx, Mb, cb, Zb));
                 pacc = pacc < 1.0 ? pacc : 1.0;
             }
-            ratio_ok = static_cast<double>(P.u_accept[item]) < pacc;        // Eq. 2
+            ratio_ok = static_cast<double>(u_accept[item]) < pacc;          // Eq. 2
         }
     }
-    return P.mode == FSD_MODE_SD ? ratio_ok : (div_ok || ratio_ok);          // Eq. 6
+    return mode == FSD_MODE_SD ? ratio_ok : (div_ok || ratio_ok);            // Eq. 6
 }
 
-template <int DT, bool VEC>
-__global__ void __launch_bounds__(512) fsd_pair_generic_kernel(PairParams P) {
-    constexpr int EPV = Logit<DT>::kPerVec;
-    __shared__ double red_d[32 * 5];
-    __shared__ float red_f[32 * 2];
+// What the three sweeps leave for the pair's final scalar work.
+struct GenericSums {
+    float Ma, Mb, ca, cb;
+    double Za, Zb, Sa, Sb, K, X;
+    bool finite;
+};
 
-    const int item = blockIdx.x;
-    const int b = item / P.G, i = item - b * P.G;
-    int trow = i;
-    if (P.parent != nullptr) {
-        const int par = P.parent[item];
-        if (par < -1 || par >= i) {
-            if (threadIdx.x == 0) {
-                P.divergence[item] = __int_as_float(0x7fc00000);
-                P.item_bits[item] = 0;
-                P.item_status[item] = FSD_ROW_BADTREE;
-            }
-            return;
-        }
-        trow = par + 1;
-    }
-    const size_t rb = static_cast<size_t>(P.V) * Logit<DT>::kBytes;
-    const char* a_row = static_cast<const char*>(P.target) + (static_cast<size_t>(b) * (P.G + 1) + trow) * rb;
-    const char* b_row = static_cast<const char*>(P.draft) + (static_cast<size_t>(b) * P.G + i) * rb;
+// The three sweeps over one pair of rows by the whole CTA; every thread returns the same sums.
+// `red_d` holds at least 32 * 5 doubles, `red_f` at least 32 * 2 floats.
+template <int DT, bool VEC>
+__device__ inline GenericSums generic_pair_sums(const char* a_row, const char* b_row, int V, int div, double* red_d, float* red_f) {
+    constexpr int EPV = Logit<DT>::kPerVec;
     const int tid = threadIdx.x, nthr = blockDim.x;
-    const int nvec = P.V / EPV;
+    const int nvec = V / EPV;
+    GenericSums r;
 
     // sweep 1: row maxima (exact)
     float mx[2] = {-INFINITY, -INFINITY};
@@ -117,7 +106,7 @@ __global__ void __launch_bounds__(512) fsd_pair_generic_kernel(PairParams P) {
             for (int e = 0; e < EPV; ++e) { mx[0] = fmaxf(mx[0], xa[e]); mx[1] = fmaxf(mx[1], xb[e]); }
         }
     } else {
-        for (int k = tid; k < P.V; k += nthr) {
+        for (int k = tid; k < V; k += nthr) {
             mx[0] = fmaxf(mx[0], load_logit<DT>(a_row, k));
             mx[1] = fmaxf(mx[1], load_logit<DT>(b_row, k));
         }
@@ -146,7 +135,7 @@ __global__ void __launch_bounds__(512) fsd_pair_generic_kernel(PairParams P) {
             for (int e = 0; e < EPV; ++e) term2(xa[e], xb[e]);
         }
     } else {
-        for (int k = tid; k < P.V; k += nthr) term2(load_logit<DT>(a_row, k), load_logit<DT>(b_row, k));
+        for (int k = tid; k < V; k += nthr) term2(load_logit<DT>(a_row, k), load_logit<DT>(b_row, k));
     }
     double s2[5] = {za, zb, sa, sb, kk};
     block_sum<5>(s2, red_d);
@@ -155,16 +144,18 @@ __global__ void __launch_bounds__(512) fsd_pair_generic_kernel(PairParams P) {
 
     // sweep 3: the sums that need both normalisers (JS: s log2 s; TV: |p - q|)
     double X = 0.0;
-    if (finite && P.div != FSD_DIV_KL) {
+    if (finite && div != FSD_DIV_KL) {
         const float ia = static_cast<float>(1.0 / Za), ib = static_cast<float>(1.0 / Zb);
-        const bool js = P.div == FSD_DIV_JS;
+        const bool js = div == FSD_DIV_JS;
         float acc = 0.f;
         auto term3 = [&](float a, float bq) {
             // explicit roundings: a fused p - q would keep one product unrounded and make TV(p, p) != 0
             const float p = __fmul_rn(ex2(fmaf(a, kLog2e, ca)), ia), q = __fmul_rn(ex2(fmaf(bq, kLog2e, cb)), ib);
             if (js) {
+                // below the normal range lg2 (which flushes its operand) would return -inf;
+                // such a term is smaller than 1e-35 and left out
                 const float s = p + q;
-                acc += s > 0.f ? s * lg2(s) : 0.f;
+                acc += s >= 1.17549435e-38f ? s * lg2(s) : 0.f;
             } else {
                 acc += fabsf(p - q);
             }
@@ -178,19 +169,50 @@ __global__ void __launch_bounds__(512) fsd_pair_generic_kernel(PairParams P) {
                 for (int e = 0; e < EPV; ++e) term3(xa[e], xb[e]);
             }
         } else {
-            for (int k = tid; k < P.V; k += nthr) term3(load_logit<DT>(a_row, k), load_logit<DT>(b_row, k));
+            for (int k = tid; k < V; k += nthr) term3(load_logit<DT>(a_row, k), load_logit<DT>(b_row, k));
         }
         double s3[1] = {acc};
         block_sum<1>(s3, red_d);
         X = s3[0];
     }
+    r.Ma = Ma; r.Mb = Mb; r.ca = ca; r.cb = cb;
+    r.Za = Za; r.Zb = Zb; r.Sa = s2[2]; r.Sb = s2[3]; r.K = s2[4]; r.X = X;
+    r.finite = finite;
+    return r;
+}
 
-    if (tid == 0) {
+template <int DT, bool VEC>
+__global__ void __launch_bounds__(512) fsd_pair_generic_kernel(PairParams P) {
+    __shared__ double red_d[32 * 5];
+    __shared__ float red_f[32 * 2];
+
+    const int item = blockIdx.x;
+    const int b = item / P.G, i = item - b * P.G;
+    int trow = i;
+    if (P.parent != nullptr) {
+        const int par = P.parent[item];
+        if (par < -1 || par >= i) {
+            if (threadIdx.x == 0) {
+                P.divergence[item] = __int_as_float(0x7fc00000);
+                P.item_bits[item] = 0;
+                P.item_status[item] = FSD_ROW_BADTREE;
+            }
+            return;
+        }
+        trow = par + 1;
+    }
+    const size_t rb = static_cast<size_t>(P.V) * Logit<DT>::kBytes;
+    const char* a_row = static_cast<const char*>(P.target) + (static_cast<size_t>(b) * (P.G + 1) + trow) * rb;
+    const char* b_row = static_cast<const char*>(P.draft) + (static_cast<size_t>(b) * P.G + i) * rb;
+    const GenericSums r = generic_pair_sums<DT, VEC>(a_row, b_row, P.V, P.div, red_d, red_f);
+
+    if (threadIdx.x == 0) {
         float D = __int_as_float(0x7fc00000);
-        if (finite) D = static_cast<float>(combine_divergence(P.div, Za, Zb, s2[2], s2[3], s2[4], X));
+        if (r.finite) D = static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X));
         P.divergence[item] = D;
-        P.item_bits[item] = accept_bit(P, item, finite, D, a_row, b_row, DT, Ma, ca, Za, Mb, cb, Zb);
-        P.item_status[item] = finite ? 0 : FSD_ROW_NONFINITE;
+        P.item_bits[item] = accept_bit(P.mode, P.cmp, P.T, P.tokens, P.u_accept, P.V, item, r.finite, D, a_row, b_row, DT,
+                                       r.Ma, r.ca, r.Za, r.Mb, r.cb, r.Zb);
+        P.item_status[item] = r.finite ? 0 : FSD_ROW_NONFINITE;
     }
 }
 
