@@ -204,14 +204,6 @@ int fsd_version(void);
  * are for attribution, not throughput.  Returns FSD_OK. */
 int fsd_set_stage_event(void *event);
 
-/* Test aid (no counterpart in the paper).  The streaming kernel's second sweep waits for the
- * statistics of a pair's other CTAs by polling a counter in the workspace; the wait is bounded,
- * and a wait that runs out makes the call return with FSD_ROW_TIMEOUT set in every row_status
- * instead of hanging.  This sets the number of polls (0 restores the default, about a second of
- * waiting); a very small number makes the wait run out on purpose, which is how the give-up
- * path is tested.  Process-wide, read when a call is made.  Returns FSD_OK. */
-int fsd_set_exchange_poll_limit(unsigned int polls);
-
 /* ---- Threshold tuning (Section "Selecting T"; Discussion, "Potential further developments") ----
  * The paper tunes T on a small development set by running FSD at candidate thresholds and
  * looking at the speed each gives, and notes that FSD's decisions are a deterministic function

@@ -8,7 +8,6 @@ from .binding import (  # noqa: F401
     fsd_default_opts,
     fsd_host_staging_bytes,
     fsd_set_stage_event,
-    fsd_set_exchange_poll_limit,
     fsd_status_string,
     fsd_threshold_sweep,
     fsd_verify_chain,

@@ -85,8 +85,6 @@ def _load():
         lib.fsd_version.restype = C.c_int
         lib.fsd_set_stage_event.argtypes = [C.c_void_p]
         lib.fsd_set_stage_event.restype = C.c_int
-        lib.fsd_set_exchange_poll_limit.argtypes = [C.c_uint]
-        lib.fsd_set_exchange_poll_limit.restype = C.c_int
         lib.fsd_threshold_sweep.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, C.c_int, vp, vp, C.c_void_p]
         lib.fsd_threshold_sweep.restype = C.c_int
         lib.fsd_calibrate_threshold.argtypes = [vp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, C.c_void_p]
@@ -134,12 +132,6 @@ def fsd_set_stage_event(event) -> int:
     if event is not None:
         handle = getattr(event, "cuda_event", event)
     return _load().fsd_set_stage_event(handle)
-
-
-def fsd_set_exchange_poll_limit(polls: int) -> int:
-    """Polls the streaming kernel's second sweep spends on a pair's counter before it gives up
-    (0: the default); a test aid."""
-    return _load().fsd_set_exchange_poll_limit(int(polls))
 
 
 def fsd_workspace_bytes(B: int, positions: int, V: int, opts: FsdOpts) -> int:

@@ -10,7 +10,7 @@
 #include "fsd_device.cuh"
 #include "fsd_finish.cuh"
 #include "fsd_pair_generic.cuh"
-#include "fsd_pair_pipeline.cuh"
+#include "fsd_pair_stream.cuh"
 #include "fsd_tuning.cuh"
 
 namespace {
@@ -24,9 +24,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 struct Workspace {
     int32_t* item_bits;
     int32_t* item_status;
-    int* flags;                // [0] = a bounded device-side wait ran out; zeroed by every call together with `arrived`
-    int* arrived;              // per pair: CTAs of the streaming kernel that have published their part
-    size_t zero_bytes;         // flags + arrived
+    int* flags;                // [0] = a bounded device-side wait ran out
     PairRecord* records;       // per-pair totals of the streaming kernel
     size_t bytes;
 };
@@ -41,9 +39,6 @@ Workspace carve(void* base, int B, int G) {
     p += align_up(items * sizeof(int32_t));
     w.flags = reinterpret_cast<int*>(p);
     p += kAlign;
-    w.arrived = reinterpret_cast<int*>(p);
-    p += align_up(items * sizeof(int));
-    w.zero_bytes = static_cast<size_t>(p - reinterpret_cast<char*>(w.flags));
     w.records = reinterpret_cast<PairRecord*>(p);
     p += align_up(items * sizeof(PairRecord));
     w.bytes = static_cast<size_t>(p - static_cast<char*>(base));
@@ -79,105 +74,87 @@ int finish_cluster_size(int B, int V) {
 }
 
 std::atomic<void*> g_stage_event{nullptr};   // see fsd_set_stage_event
-std::atomic<uint32_t> g_poll_limit{kPollLimit};   // see fsd_set_exchange_poll_limit
 
 // ---- streaming kernel launch -----------------------------------------------------------
 constexpr int kMaxDev = 64;
 
-// Number of SMs of the current device (cached), or 0.
-int sm_count() {
-    static std::atomic<int> cached[kMaxDev] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return 0;
-    int n = cached[dev].load();
-    if (n == 0) {
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        cached[dev].store(n);
-    }
-    return n;
-}
-
-// CTAs per pair for the streaming kernel: a CTA's slice must leave the tensor-memory ring at
-// least two chunks of slack (so that the first sweep of the next pair can start while the
-// statistics of this one travel); among the sizes that do, the one with the least estimated
-// time, rounds * (slice + a fixed cost per round).  0 if the shape is not eligible (the generic
-// kernel takes it).
-int pipeline_group(int nvec_row, int n_items, int sms, int chunks, bool vec) {
-    if (!vec || nvec_row < 64 || sms < 1) return 0;
-    int best = 0;
-    long long best_cost = 0;
-    for (int g = 1; g <= kMaxGroup && g <= sms; ++g) {
-        const int slice = (nvec_row + g - 1) / g;
-        const int ns = (slice + kStageVecs - 1) / kStageVecs;
-        if (ns > chunks - 2) continue;
-        const int groups = sms / g;
-        const long long rounds = (n_items + groups - 1) / groups;
-        const long long cost = rounds * (slice + 600);
-        if (best == 0 || cost < best_cost) { best = g; best_cost = cost; }
-    }
-    return best;
-}
-
 template <int DT, int DIV>
-int prepare_pipeline() {
-    static std::atomic<int> ready[kMaxDev] = {};
+int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
+    static int max_clusters[kMaxDev][5] = {};       // per device, per log2(C); 0 = not yet queried
+    static std::mutex mu;
+    auto kernel = fsd_pair_stream_kernel<DT, DIV>;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return FSD_ERR_CUDA;
-    if (ready[dev].load() == 0) {
-        if (cudaFuncSetAttribute(fsd_pair_pipeline_kernel<DT, DIV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kPipeSmemBytes)) != cudaSuccess)
-            return FSD_ERR_CUDA;
-        ready[dev].store(1);
+    int lc = 0;
+    while ((1 << lc) < C) ++lc;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.dynamicSmemBytes = kStreamSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int nclus;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (max_clusters[dev][lc] == 0) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+                return FSD_ERR_CUDA;
+            if (cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+                return FSD_ERR_CUDA;
+            if (C > 8) {                            // above the portable cluster size: opt in
+                if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+                    cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+                    return FSD_ERR_CUDA;
+            }
+            cfg.gridDim = dim3(C, 1, 1);
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, fsd_stream_occupancy_twin, &cfg) != cudaSuccess || n < 1)
+                return FSD_ERR_CUDA;
+            max_clusters[dev][lc] = n;
+        }
+        nclus = max_clusters[dev][lc];
     }
+    if (nclus > sp.n_items) nclus = sp.n_items;
+    cfg.gridDim = dim3(static_cast<unsigned>(nclus) * C, 1, 1);
+    if (cudaLaunchKernelEx(&cfg, kernel, sp) != cudaSuccess) return FSD_ERR_CUDA;
     return FSD_OK;
 }
 
-// The CTAs of a group wait for one another, so all of them must be resident at once: a
-// cooperative launch, which the runtime refuses when the grid does not fit.
-template <int DT, int DIV>
-int launch_pipeline(const PipeParams& pp, int n_groups, cudaStream_t s) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(n_groups) * pp.group, 1, 1);
-    cfg.blockDim = dim3(kPipeThreads, 1, 1);
-    cfg.dynamicSmemBytes = kPipeSmemBytes;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, fsd_pair_pipeline_kernel<DT, DIV>, pp) != cudaSuccess) return FSD_ERR_CUDA;
-    return FSD_OK;
+// Cluster size for the streaming kernel: the smallest power of two whose per-CTA slice fits
+// on chip; 0 if the shape is not eligible (the generic kernel takes it).
+int stream_cluster_size(int nvec_row, bool vec) {
+    if (!vec || nvec_row < 64) return 0;
+    for (int C = 1; C <= kStreamMaxCluster; C <<= 1)
+        if ((nvec_row + C - 1) / C <= kMaxVecPerCta) return C;
+    return 0;
 }
 
 template <int DT>
-int launch_all(const PairParams& pp, FinishParams fp, bool vec, const Workspace& ws, cudaStream_t s) {
+int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, PairRecord* records, cudaStream_t s) {
     const int items = pp.B * pp.G;
     const int nvec_row = pp.V / Logit<DT>::kPerVec;
-    constexpr int kChunks = kTmemCols / (kS1PerQuarter * kVecPerThread * 2 * Logit<DT>::kPerVec);
-    const int sms = sm_count();
-    const int group = pipeline_group(nvec_row, items, sms, kChunks, vec);
-    if (group > 0) {
-        PipeParams sp;
+    const int C = stream_cluster_size(nvec_row, vec);
+    if (C > 0) {
+        StreamParams sp;
         sp.target = pp.target; sp.draft = pp.draft; sp.parent = pp.parent; sp.B = pp.B; sp.G = pp.G;
-        sp.nvec_row = nvec_row; sp.n_items = items; sp.group = group; sp.records = ws.records;
-        sp.arrived = ws.arrived; sp.timeout_flag = ws.flags; sp.poll_limit = g_poll_limit.load();
-        int n_groups = sms / group;
-        if (n_groups > items) n_groups = items;
-        // everything that can fail without a launch comes before the first thing put on the stream
+        sp.nvec_row = nvec_row; sp.n_items = items; sp.records = records; sp.timeout_flag = flags; sp.next_pair = flags + 1;
+        // the flag block starts every call at zero: [0] timeout, [1] pairs handed out
+        if (cudaMemsetAsync(flags, 0, kAlign, s) != cudaSuccess) return FSD_ERR_CUDA;
         int rc;
-        if (pp.div == FSD_DIV_JS)      rc = prepare_pipeline<DT, FSD_DIV_JS>();
-        else if (pp.div == FSD_DIV_KL) rc = prepare_pipeline<DT, FSD_DIV_KL>();
-        else                           rc = prepare_pipeline<DT, FSD_DIV_TV>();
+        if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, C, s);
+        else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, C, s);
+        else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, C, s);
         if (rc != FSD_OK) return rc;
-        // the timeout flag and the pairs' counters start every call at zero
-        if (cudaMemsetAsync(ws.flags, 0, ws.zero_bytes, s) != cudaSuccess) return FSD_ERR_CUDA;
-        if (pp.div == FSD_DIV_JS)      rc = launch_pipeline<DT, FSD_DIV_JS>(sp, n_groups, s);
-        else if (pp.div == FSD_DIV_KL) rc = launch_pipeline<DT, FSD_DIV_KL>(sp, n_groups, s);
-        else                           rc = launch_pipeline<DT, FSD_DIV_TV>(sp, n_groups, s);
-        if (rc != FSD_OK) return rc;
-        fp.timeout_flag = ws.flags;
-        fp.records = ws.records;
+        fp.timeout_flag = flags;
+        fp.records = records;
     } else {
         if (vec) fsd_pair_generic_kernel<DT, true><<<items, 512, 0, s>>>(pp);
         else     fsd_pair_generic_kernel<DT, false><<<items, 512, 0, s>>>(pp);
@@ -243,7 +220,8 @@ int verify_common(const void* target, const void* draft, const int32_t* tokens, 
     const bool vec = (static_cast<size_t>(V) * es) % 16 == 0 && aligned(target, 16) && aligned(draft, 16);
     fp.vec = vec ? 1 : 0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, ws, s) : launch_all<FSD_F32>(pp, fp, vec, ws, s);
+    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, ws.flags, ws.records, s)
+                                       : launch_all<FSD_F32>(pp, fp, vec, ws.flags, ws.records, s);
 }
 
 struct HostStaging {
@@ -441,11 +419,6 @@ int fsd_version(void) { return 100; }
 
 int fsd_set_stage_event(void* event) {
     g_stage_event.store(event);
-    return FSD_OK;
-}
-
-int fsd_set_exchange_poll_limit(unsigned int polls) {
-    g_poll_limit.store(polls == 0 ? kPollLimit : polls);
     return FSD_OK;
 }
 

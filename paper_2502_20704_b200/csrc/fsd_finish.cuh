@@ -9,20 +9,19 @@
 // exponentials and partial sums of step 3 are double precision: each thread owns a contiguous
 // chunk of the vocabulary, chunk sums are combined by a fixed-order scan (thread -> warp ->
 // CTA -> cluster), and the first thread whose inclusive sum exceeds u * total re-walks its
-// chunk.  The double exponential is a 256-entry table times a degree-4 polynomial (about ten
+// chunk.  The double exponential is a 64-entry table times a degree-5 polynomial (about ten
 // fp64 operations); the rows involved are a 1/(2*gamma+1) share of all logits.
 #pragma once
 
 #include "fsd_device.cuh"
 #include "fsd_pair_generic.cuh"
-#include "fsd_pair_pipeline.cuh"
+#include "fsd_pair_stream.cuh"
 
 namespace fsd {
 
 constexpr int kFinishThreads = 512;
 constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kMaxTreeNodes = 1024;
-constexpr int kBitRedo = -2;                 // item_bits value of a pair that awaits the exact recomputation
 
 struct FinishParams {
     const void* target;        // [B, G+1, V]
@@ -57,7 +56,7 @@ struct FinishShared {
     double gather_d[kMaxClusterSize];   // one value per CTA of the cluster (see cluster_gather)
     int gather_i[kMaxClusterSize];
     double exp_table[kExpTable];   // 2^(j/256)
-    double red_d[32 * 5];
+    double red_d[32 * 2];
     float red_f[32 * 2];
     double warp_tot[32];
     int cand;                  // lowest thread whose inclusive sum exceeds the target
@@ -66,7 +65,6 @@ struct FinishShared {
     int row_sel;               // target row the token is drawn from
     int n_acc;
     int bad;
-    int n_redo;                // pairs of this row whose record asks for the exact recomputation
     int16_t tree_depth[kMaxTreeNodes];
     int8_t tree_ok[kMaxTreeNodes];
     int8_t tree_bit[kMaxTreeNodes];
@@ -130,15 +128,15 @@ struct PairTotals {
 __device__ __forceinline__ double pow2_int_d(double d) {
     return d < -1022.0 ? 0.0 : __hiloint2double((1023 + static_cast<int>(d)) << 20, 0);
 }
-__device__ __forceinline__ double group_sum(double v) {       // over the kMaxGroup lanes of a record
+__device__ __forceinline__ double group_sum(double v) {       // over the kStreamMaxCluster lanes of a record
 #pragma unroll
-    for (int m = kMaxGroup / 2; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
     return v;
 }
 // Called by all 32 lanes: lane 16*q + r folds part r of the record `rec` of group q (null: no
 // record for this group); every lane of a group returns the group's totals.
 __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
-    const int r = threadIdx.x & (kMaxGroup - 1);
+    const int r = threadIdx.x & (kStreamMaxCluster - 1);
     PairTotals t;
     Stats c;
     c.ka = -INFINITY; c.kb = -INFINITY; c.za = 0.f; c.zb = 0.f; c.s0 = 0.f; c.sb = 0.f; c.x = 0.f; c.diff = 0;
@@ -146,7 +144,7 @@ __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     if (rec != nullptr && r < static_cast<int>(rec->ncta)) { c = rec->part[r]; x = rec->x[r]; }
     float ka = c.ka, kb = c.kb;                          // NaN references win
 #pragma unroll
-    for (int m = kMaxGroup / 2; m > 0; m >>= 1) {
+    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) {
         const float oa = __shfl_xor_sync(0xffffffffu, ka, m), ob = __shfl_xor_sync(0xffffffffu, kb, m);
         ka = (oa != oa || ka != ka) ? __int_as_float(0x7fc00000) : fmaxf(ka, oa);
         kb = (ob != ob || kb != kb) ? __int_as_float(0x7fc00000) : fmaxf(kb, ob);
@@ -171,22 +169,20 @@ __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     t.X = group_sum(static_cast<double>(x));
     uint32_t df = c.diff;
 #pragma unroll
-    for (int m = kMaxGroup / 2; m > 0; m >>= 1) df |= __shfl_xor_sync(0xffffffffu, df, m);
+    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) df |= __shfl_xor_sync(0xffffffffu, df, m);
     t.differ = df;
     return t;
 }
 
-// Returns false (and leaves the outputs alone) when the record asks for the exact recomputation.
-__device__ inline bool judge_record(const FinishParams& P, int item, const PairTotals& r, const void* a_row, const void* b_row, int dt,
+__device__ inline void judge_record(const FinishParams& P, int item, const PairTotals& r, const void* a_row, const void* b_row, int dt,
                                     float& D_out, int& bit_out, int& st_out) {
     if (P.records[item].state & kRecordBadTree) {
         D_out = __int_as_float(0x7fc00000); bit_out = 0; st_out = FSD_ROW_BADTREE;
-        return true;
+        return;
     }
-    if (r.differ & kDiffRedo) return false;
     const bool finite = isfinite(r.ka) && isfinite(r.kb) && r.Za > 0.0 && r.Zb > 0.0 && isfinite(r.Za) && isfinite(r.Zb);
     float D = __int_as_float(0x7fc00000);
-    if (finite) D = (r.differ & kDiffRows) ? static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X)) : 0.0f;
+    if (finite) D = r.differ ? static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X)) : 0.0f;
     const bool div_ok = finite && passes(D, P.T, P.cmp);
     int bit = div_ok;
     if (P.mode != FSD_MODE_FSD) {
@@ -212,7 +208,6 @@ __device__ inline bool judge_record(const FinishParams& P, int item, const PairT
         bit = P.mode == FSD_MODE_SD ? ratio_ok : (div_ok || ratio_ok);          // Eq. 6
     }
     D_out = D; bit_out = bit; st_out = finite ? 0 : FSD_ROW_NONFINITE;
-    return true;
 }
 
 // Calls f(k, a_k, b_k) for k in [k0, k1) in order; 16-byte loads when `vec` (then k0 is a
@@ -252,7 +247,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const char* d_base = static_cast<const char*>(P.draft) + static_cast<size_t>(b) * G * rb;
     const bool tree = P.parent != nullptr;
 
-    if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.n_redo = 0; sh.row_sel = 0; sh.token = -1; }
+    if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; sh.token = -1; }
     if (tid < kExpTable) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / kExpTable));
     __syncthreads();
     // everything above touched no global memory; what follows reads what the pair kernel wrote
@@ -274,16 +269,11 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                 }
                 float D;
                 int bit, s;
-                if (judge_record(P, item, tot, t_base + static_cast<size_t>(trow) * rb, d_base + static_cast<size_t>(i) * rb, DT, D, bit, s)) {
-                    if (rank == 0) P.divergence[item] = D;
-                    P.item_bits[item] = bit;             // every CTA of the cluster writes the same value
-                    st |= s;
-                    if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
-                    else if (!bit && i < first) first = i;
-                } else {
-                    P.item_bits[item] = kBitRedo;
-                    atomicAdd(&sh.n_redo, 1);
-                }
+                judge_record(P, item, tot, t_base + static_cast<size_t>(trow) * rb, d_base + static_cast<size_t>(i) * rb, DT, D, bit, s);
+                if (rank == 0) P.divergence[item] = D;
+                st |= s;
+                if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
+                else if (!bit && i < first) first = i;
             }
         }
     } else {
@@ -303,34 +293,6 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         if (!tree) atomicMin(&sh.n_acc, first);
     }
     __syncthreads();
-    if (sh.n_redo > 0) {
-        // Pairs whose streamed sums left the range of their references (a logit far above the
-        // first ones met, a NaN, +inf): the whole CTA recomputes them with exact maxima.
-        for (int i = 0; i < G; ++i) {
-            const int item = b * G + i;
-            if (P.item_bits[item] != kBitRedo) continue;     // uniform over the CTA
-            int trow = i;
-            if (tree) {
-                const int par = P.parent[item];
-                trow = (par >= -1 && par < i) ? par + 1 : 0;
-            }
-            const char* ar = t_base + static_cast<size_t>(trow) * rb;
-            const char* br = d_base + static_cast<size_t>(i) * rb;
-            const GenericSums r = P.vec ? generic_pair_sums<DT, true>(ar, br, V, P.div, sh.red_d, sh.red_f)
-                                        : generic_pair_sums<DT, false>(ar, br, V, P.div, sh.red_d, sh.red_f);
-            if (tid == 0) {
-                float D = __int_as_float(0x7fc00000);
-                if (r.finite) D = static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X));
-                const int bit = accept_bit(P.mode, P.cmp, P.T, P.tokens, P.u_accept, V, item, r.finite, D, ar, br, DT,
-                                           r.Ma, r.ca, r.Za, r.Mb, r.cb, r.Zb);
-                if (rank == 0) P.divergence[item] = D;
-                if (!r.finite) sh.bad |= FSD_ROW_NONFINITE;
-                if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
-                else if (!bit && i < sh.n_acc) sh.n_acc = i;
-            }
-        }
-        __syncthreads();
-    }
 
     // ---- 2. accepted prefix (chain) or deepest accepted path (tree) ----
     if (tid == 0) {
@@ -394,9 +356,9 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             if (r->state & kRecordStats) {                // any common reference near the maximum serves
                 float rka = -INFINITY;
                 bool nan = false;
-                for (uint32_t c = 0; c < r->ncta && c < kMaxGroup; ++c) {
+                for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
                     const float a = r->part[c].ka;
-                    nan = nan || a != a || (r->part[c].diff & kDiffRedo) != 0;   // out-of-range sums: the reference is no guide
+                    nan = nan || a != a;
                     rka = fmaxf(rka, a);
                 }
                 if (!nan && isfinite(rka)) { kref = rka; have_ref = true; }
@@ -520,9 +482,9 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         if (r->state & kRecordStats) {
             float fa = -INFINITY, fb = -INFINITY;
             bool nan = false;
-            for (uint32_t c = 0; c < r->ncta && c < kMaxGroup; ++c) {
+            for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
                 const float a = r->part[c].ka, q = r->part[c].kb;
-                nan = nan || a != a || q != q || (r->part[c].diff & kDiffRedo) != 0;
+                nan = nan || a != a || q != q;
                 fa = fmaxf(fa, a); fb = fmaxf(fb, q);
             }
             if (!nan && isfinite(fa) && isfinite(fb)) { kra = fa; krb = fb; common = true; }

@@ -51,6 +51,10 @@ def test_config3_zipf_with_disjoint_drafts():
     assert c.disjoint.any()
     r = _check(c, div="kl", T=0.3)
     r = _check(c, div="tv", T=0.3)
+    # the strict and the relaxed ratio rule (Eq. 1-3, Eq. 6) at a full LLM vocabulary
+    _check(c, mode="sd")
+    _check(c, mode="rfsd", T=0.1)
+    _check(c, mode="sd", sample="greedy")
 
 
 def test_config4_headline_shape():
@@ -59,6 +63,36 @@ def test_config4_headline_shape():
     assert r["max_err"] <= 1e-4
     assert len(set(r["accept_len"].tolist())) > 2                    # the workload is not degenerate
     _check(c, T=0.2, cmp="le")
+    _check(c, div="kl", T=0.2)
+    _check(c, div="tv", T=0.2)
+    _check(c, mode="sd")
+
+
+@pytest.mark.parametrize("gamma", [10, 15, 20])
+def test_paper_candidate_lengths_at_a_full_vocabulary(gamma):
+    """The candidate lengths the paper runs (Appendix F: 5, 10, 15, 20) on the headline vocabulary;
+    a small batch keeps the oracle affordable."""
+    c = gi.make_chain(3, gamma, 152064, dtype="bf16", recipe="zipf", sigma=(0.2, 2.0), sigma_mode="uniform",
+                      disjoint_frac=0.1, workload_id=400 + gamma)
+    r = _check(c, T=0.2)
+    assert r["max_err"] <= 1e-4
+    _check(c, mode="sd")
+    _check(c, mode="rfsd", T=0.2)
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 32776), ("f32", 16388), ("bf16", 65544), ("bf16", 131080)])
+def test_slices_of_unequal_stage_counts_within_a_cluster(dtype, V):
+    """Row lengths that split over the cluster into slices of which some need one ring stage more
+    than the others, with more pairs than the clusters take in their first rounds: the CTAs of a
+    cluster must still agree on which pair comes next."""
+    c = gi.make_chain(16, 8, V, dtype=dtype, recipe="zipf", sigma=(0.2, 1.5), sigma_mode="uniform",
+                      disjoint_frac=0.1, workload_id=420)
+    r = _check(c, T=0.2)
+    assert not (r["gpu"].row_status & 2).any()
+    _check(c, div="tv", T=0.3)
+    if V == 32776:
+        t = gi.make_tree(4, 40, V, dtype=dtype, sigma=0.6, max_depth=5, workload_id=421)
+        parity.check_tree(t, T=0.1)
 
 
 def test_config5_tree():
