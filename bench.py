@@ -1,15 +1,22 @@
 #!/usr/bin/env python
 """Benchmark of the batched FSD verification step.
 
-One "step" is one fsd_verify_chain call (every kernel of the hot path) over one batch of
-synthetic logits of the headline workload: chain, B=64, gamma=8, V=152064, bf16, JS, T=0.2.
-Prints ONE JSON line.  `value` is verified draft positions per second with inputs resident in
-HBM; `e2e` is the same through the host-buffer entry point with the copies inside the timed
-region; `roofline` relates the algorithmic bytes (each needed logit read once) to the measured
-HBM copy bandwidth; `cpu_baseline` times the double-precision CPU oracle on a bounded sample.
+One "step" is one verify call (every kernel of the hot path: fsd_verify_chain, or fsd_verify_tree
+for the tree workload) over one batch of synthetic logits.  With no flags the workload is the
+headline one: chain, B=64, gamma=8, V=152064, bf16, JS, T=0.2 ("c4").  Prints ONE JSON line.
+`value` is verified draft positions per second with inputs resident in HBM; `e2e` is the same
+with host buffers in and host results out, the copies inside the timed region; `roofline` relates
+the dominant kernel's algorithmic bytes (each needed logit read once) to the measured HBM copy
+bandwidth, with the whole call beside it; `cpu_baseline` times the double-precision CPU oracle
+on a bounded sample of the same workload (all cores and one core) and `parity` compares the timed
+call's results with that oracle run.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload c1|c2|c3|c4|c5] [--div js|kl|tv] [--mode fsd|sd|rfsd]
+                  [--V n] [--gamma n] [--B n] [--dtype bf16|f32]
 
+Inputs smaller than a third of three L2 sizes are replicated until the rotating set is three L2
+sizes; the time with a single copy (served from L2) is reported separately as `hot_l2`.
 With N > 1 (under torchrun) every rank runs an independent replica of the workload on its own
 GPU (the path has no exchange step), the timed region is bracketed by barriers and the time is
 the maximum over ranks.
@@ -32,13 +39,14 @@ if ROOT not in sys.path:
 
 import fsd_inputs as gi  # noqa: E402
 
-WORKLOAD = "c4"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + written) of one pair-kernel launch on the headline workload, from the ncu
-# capture summarised under profiles/; set to None whenever that kernel changes after the capture.
+# capture summarised under profiles/; None whenever that kernel has changed since the capture.
 PAIR_KERNEL_DRAM_BYTES = 311_719_936
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
+D_BAND = 1e-5          # |D_oracle - T| below this: the fp32 and fp64 decisions may differ
+SAMPLE_BAND = 1e-6     # a drawn token may be a neighbour when u*W is this close (times W) to an interval end
 
 
 def measured_hbm_peak():
@@ -61,7 +69,7 @@ def aggregate_over_ranks(local_ms: float, local_units: float, world: int, reduce
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read only)."""
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -124,39 +132,120 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def oracle_sample_rate(c, rows: int, T: float, nthreads: int = 0):
-    """Times the CPU oracle (as it stands) on the first `rows` batch rows; returns (positions/s, seconds, cores)."""
+# ----------------------------------------------------------------------------------------------
+# workload description
+# ----------------------------------------------------------------------------------------------
+def is_tree(c) -> bool:
+    return hasattr(c, "parent")
+
+
+def positions_per_call(c) -> int:
+    return c.B * (c.N if is_tree(c) else c.gamma)
+
+
+def input_bytes(c) -> int:
+    return int(c.target.nbytes + c.draft.nbytes)
+
+
+def describe(c, name: str, div: str, mode: str, T: float, rows=None, named=True):
+    """The `config` object of the JSON line.  `rows`: batch rows of a sample (reference arm)."""
+    B = c.B if rows is None else rows
+    if is_tree(c):
+        shape = f"tree FSD verify B={B} N={c.N} V={c.V} {c.dtype}"
+        dims = {"B": B, "N": c.N, "V": c.V, "max_depth": c.max_depth}
+    else:
+        shape = f"chain FSD verify B={B} gamma={c.gamma} V={c.V} {c.dtype}"
+        dims = {"B": B, "gamma": c.gamma, "V": c.V}
+    tag = f"config {name[1:]}" if named else f"config {name[1:]}'s recipe, other shape"
+    if rows is not None:
+        tag = f"{rows}-row sample of config {name[1:]}'s recipe"
+    cfg = {"workload": f"{shape} {div.upper()} T={T:g} mode={mode} ({tag})", **dims, "logit_dtype": c.dtype,
+           "divergence": div, "mode": mode, "threshold": T, "parallelism": "independent replicas"}
+    return cfg
+
+
+def oracle_run(c, rows: int, div: str, mode: str, T: float, nthreads: int = 0, band: float = SAMPLE_BAND):
+    """One run of the CPU oracle (as it stands) on the first `rows` batch rows; returns (result, seconds)."""
     from oracle import fsd_oracle as orc
     orc.lib()
-    cores = orc.max_threads() if nthreads <= 0 else nthreads
     t0 = time.perf_counter()
-    orc.verify_chain(c.target[:rows], c.draft[:rows], None, None, c.u_sample[:rows], dtype=c.dtype, div="js",
-                     mode="fsd", T=T, nthreads=nthreads)
-    dt = time.perf_counter() - t0
-    return rows * c.gamma / dt, dt, cores
+    if is_tree(c):
+        r = orc.verify_tree(c.target[:rows], c.draft[:rows], c.parent[:rows], c.u_sample[:rows], c.max_depth,
+                            dtype=c.dtype, div=div, T=T, band=band, nthreads=nthreads)
+    else:
+        r = orc.verify_chain(c.target[:rows], c.draft[:rows], c.draft_tokens[:rows], c.u_accept[:rows],
+                             c.u_sample[:rows], dtype=c.dtype, div=div, mode=mode, T=T, band=band, nthreads=nthreads)
+    return r, time.perf_counter() - t0
 
 
-def run_reference(args, rank: int, world: int):
+def oracle_rate(c, rows: int, div: str, mode: str, T: float, nthreads: int, budget_s: float):
+    """Positions per second of the oracle on `rows` batch rows, repeated for about `budget_s` seconds."""
+    per_row = positions_per_call(c) // c.B
+    _, secs = oracle_run(c, rows, div, mode, T, nthreads)
+    reps = int(min(50, max(1, budget_s / max(secs, 1e-4)))) if secs < budget_s / 2 else 0
+    if reps:
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            oracle_run(c, rows, div, mode, T, nthreads)
+        secs = (time.perf_counter() - t0) / reps
+    return rows * per_row / secs
+
+
+def sample_rows(c) -> int:
+    """Batch rows of the oracle sample: all of a small workload, 16 of a large one."""
+    per_row_logits = (2 * (c.N if is_tree(c) else c.gamma) + 1) * c.V
+    return int(max(1, min(c.B, 16 if per_row_logits > 1_000_000 else c.B)))
+
+
+def parity_counts(c, o, rows, res, T, tol):
+    """Compares the timed call's outputs (dict of numpy arrays) with the oracle's on the sampled rows."""
+    D_g, D_o = res["D"][:rows].astype(np.float64), o.divergence
+    fin = np.isfinite(D_o)
+    same_nan = bool(np.array_equal(np.isnan(D_g), np.isnan(D_o)) and np.array_equal(np.isposinf(D_g), np.isposinf(D_o)))
+    max_err = float(np.abs(D_g[fin] - D_o[fin]).max()) if fin.any() else 0.0
+    with np.errstate(invalid="ignore"):
+        in_band = np.abs(D_o - float(np.float32(T))) < D_BAND
+    band_rows = len_mismatch = tok_other = tok_outside = 0
+    for b in range(rows):
+        affected = bool(in_band[b].any())
+        band_rows += affected
+        if res["acc"][b] != o.accept_len[b]:
+            len_mismatch += 0 if affected else 1
+            continue
+        if res["tok"][b] != o.next_token[b]:
+            tok_other += 1
+            tok_outside += 0 if o.tok_lo[b] <= res["tok"][b] <= o.tok_hi[b] else 1
+    out = {"rows_checked": rows, "max_abs_D_err": max_err, "D_tolerance": tol, "nan_inf_pattern_equal": same_nan,
+           "rows_with_D_within_1e-5_of_T": int(band_rows), "accept_len_mismatches_outside_that_band": int(len_mismatch),
+           "tokens_differing_from_oracle": int(tok_other), "of_which_outside_the_1e-6_sample_band": int(tok_outside)}
+    ok = same_nan and max_err <= tol and len_mismatch == 0 and tok_outside == 0
+    return out, ok
+
+
+def run_reference(args, rank: int):
     """The reference arm: the CPU oracle on the host cores, each step a bounded sample of the workload."""
     if rank != 0:
         return
-    rows = args.ref_rows
-    c = gi.make_config(WORKLOAD, B=rows)
-    T = float(gi.CONFIGS[WORKLOAD].thresholds[0])
+    from oracle import fsd_oracle as orc
+    name = args.workload
+    spec = gi.CONFIGS[name]
+    rows = min(args.ref_rows, spec.params["B"])
+    c = gi.make_config(name, B=rows)
+    T = float(args.T if args.T is not None else spec.thresholds[len(spec.thresholds) // 2])
     for _ in range(max(args.warmup, 1)):
-        oracle_sample_rate(c, rows, T)
+        oracle_run(c, rows, args.div, args.mode, T)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_sample_rate(c, rows, T)
+        oracle_run(c, rows, args.div, args.mode, T)
     dt = time.perf_counter() - t0
-    from oracle import fsd_oracle as orc
-    value = rows * c.gamma * args.steps / dt
-    sample = f"first {rows} of 64 batch rows of the workload per step ({rows * c.gamma} positions)"
+    units = positions_per_call(c)
+    value = units * args.steps / dt
+    sample = f"{rows} batch rows of config {name[1:]}'s recipe per step ({units} positions)"
     line = {
         "impl": "reference", "metric": "verified draft positions/sec", "value": value, "unit": "positions/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(c, rows, sampled=True),
+        "config": describe(c, name, args.div, args.mode, T, rows=rows),
         "cpu_baseline": {"value": value, "unit": "positions/s", "cores": orc.max_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": "positions/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -165,31 +254,25 @@ def run_reference(args, rank: int, world: int):
     print(json.dumps(line))
 
 
-def workload_config(c, B, sampled=False):
-    spec = gi.CONFIGS[WORKLOAD].params
-    same = (B if not sampled else spec["B"], c.gamma, c.V, c.dtype) == (spec["B"], spec["gamma"], spec["V"], spec["dtype"])
-    mb = c.elem_size * B * (2 * c.gamma + 1) * c.V / 1e6
-    return {"workload": f"chain FSD verify B={B} gamma={c.gamma} V={c.V} {c.dtype} JS T=0.2 "
-                        + ("(config 4)" if same else "(config 4's recipe, other shape)"),
-            "B": B, "gamma": c.gamma, "V": c.V, "divergence": "js", "mode": "fsd", "threshold": 0.2,
-            "parallelism": "independent replicas",
-            "l2": f"inputs ({mb:.0f} MB) exceed L2 (126 MB); 3 input copies rotated between steps"}
-
-
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=sorted(gi.CONFIGS))
+    ap.add_argument("--div", default="js", choices=["js", "kl", "tv"])
+    ap.add_argument("--mode", default="fsd", choices=["fsd", "sd", "rfsd"])
+    ap.add_argument("--T", type=float, default=None, help="threshold (default: the workload's)")
     ap.add_argument("--e2e-steps", type=int, default=12)
-    ap.add_argument("--copies", type=int, default=3)
+    ap.add_argument("--copies", type=int, default=0, help="input copies rotated between steps (0: enough for three L2 sizes)")
     ap.add_argument("--ref-rows", type=int, default=16, help="batch rows per step of the reference arm")
-    # extra rows (not the headline): the headline recipe with another vocabulary, length, batch or dtype
-    ap.add_argument("--V", type=int, default=None, help="vocabulary size instead of 152064 (e.g. 256000)")
-    ap.add_argument("--gamma", type=int, default=None, help="candidate length instead of 8 (e.g. 10, 15, 20)")
-    ap.add_argument("--B", type=int, default=None, help="batch rows instead of 64")
-    ap.add_argument("--dtype", default=None, choices=["bf16", "f32"], help="logit type instead of bf16")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle legs (cpu_baseline, parity)")
+    # other shapes with the workload's recipe (not the named configuration)
+    ap.add_argument("--V", type=int, default=None, help="vocabulary size (e.g. 256000)")
+    ap.add_argument("--gamma", type=int, default=None, help="candidate length (e.g. 10, 15, 20)")
+    ap.add_argument("--B", type=int, default=None, help="batch rows")
+    ap.add_argument("--dtype", default=None, choices=["bf16", "f32"], help="logit type")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -198,7 +281,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
     if args.impl == "reference":
-        run_reference(args, rank, world)
+        run_reference(args, rank)
         return
 
     import torch
@@ -232,56 +315,102 @@ def main():
         return float(t.item())
 
     # ---- workload (same seeded inputs on every rank: replicas) ----
+    name = args.workload
+    spec = gi.CONFIGS[name]
     overrides = {k: v for k, v in (("V", args.V), ("gamma", args.gamma), ("B", args.B), ("dtype", args.dtype))
                  if v is not None}
-    headline = not overrides
-    c = gi.make_config(WORKLOAD, **overrides)
-    T = float(gi.CONFIGS[WORKLOAD].thresholds[0])
-    B, gamma, V = c.B, c.gamma, c.V
-    opts = fsd.make_opts(div="js", mode="fsd", cmp="lt", sample="invcdf", dtype=c.dtype, T=T)
-    if c.dtype == "bf16":
-        h_target = torch.from_numpy(c.target.view(np.int16)).view(torch.bfloat16).pin_memory()
-        h_draft = torch.from_numpy(c.draft.view(np.int16)).view(torch.bfloat16).pin_memory()
-    else:
-        h_target = torch.from_numpy(c.target).pin_memory()
-        h_draft = torch.from_numpy(c.draft).pin_memory()
-    h_us = torch.from_numpy(c.u_sample).pin_memory()
-    copies = [(h_target.cuda(), h_draft.cuda()) for _ in range(max(args.copies, 1))]
+    if spec.kind == "tree" and "gamma" in overrides:
+        overrides["N"] = overrides.pop("gamma")
+    c = gi.make_config(name, **overrides)
+    tree = is_tree(c)
+    if tree and args.mode != "fsd":
+        raise SystemExit("the tree workload has the FSD rule only")
+    T = float(args.T if args.T is not None else spec.thresholds[len(spec.thresholds) // 2])
+    headline = name == "c4" and not overrides and args.div == "js" and args.mode == "fsd" and args.T is None
+    B, V = c.B, c.V
+    P = c.N if tree else c.gamma                      # positions per batch row
+    units = positions_per_call(c)
+    opts = fsd.make_opts(div=args.div, mode=args.mode, cmp="lt", sample="invcdf", dtype=c.dtype, T=T)
+
+    def pinned(a):
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+        return torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+
+    h_target, h_draft, h_us = pinned(c.target), pinned(c.draft), pinned(c.u_sample)
+    h_tok = pinned(c.draft_tokens) if not tree else None
+    h_ua = pinned(c.u_accept) if not tree else None
+    h_par = pinned(c.parent.astype(np.int32)) if tree else None
+    in_bytes = input_bytes(c)
+    n_copies = args.copies if args.copies > 0 else int(min(512, max(3, -(-3 * L2_BYTES // in_bytes))))
+    copies = [(h_target.cuda(), h_draft.cuda()) for _ in range(n_copies)]
     us = h_us.cuda()
+    tokd = h_tok.cuda() if h_tok is not None else None
+    uad = h_ua.cuda() if h_ua is not None else None
+    pard = h_par.cuda() if h_par is not None else None
     acc = torch.empty(B, dtype=torch.int32, device="cuda")
     tok = torch.empty(B, dtype=torch.int32, device="cuda")
-    D = torch.empty(B, gamma, dtype=torch.float32, device="cuda")
+    D = torch.empty(B, P, dtype=torch.float32, device="cuda")
     st = torch.empty(B, dtype=torch.int32, device="cuda")
-    wsb = fsd.fsd_workspace_bytes(B, gamma, V, opts)
+    path = torch.empty(B, c.max_depth, dtype=torch.int32, device="cuda") if tree else None
+    wsb = fsd.fsd_workspace_bytes(B, P, V, opts)
     ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
     sptr = stream.cuda_stream
-    launches_per_step = 2
+    launches_per_step = 2                              # pair kernel + finish kernel (the flag memset is not a kernel of this library)
 
-    def step(i):
-        t, d = copies[i % len(copies)]
-        rc = fsd.fsd_verify_chain(t, d, None, None, us, B, gamma, V, opts, acc, tok, D, st, ws, wsb, sptr)
+    def call(t, d):
+        if tree:
+            rc = fsd.fsd_verify_tree(t, d, pard, us, B, P, V, c.max_depth, opts, acc, path, tok, D, st, ws, wsb, sptr)
+        else:
+            rc = fsd.fsd_verify_chain(t, d, tokd, uad, us, B, P, V, opts, acc, tok, D, st, ws, wsb, sptr)
         if rc != 0:
             raise RuntimeError(fsd.fsd_status_string(rc))
 
+    def step(i):
+        call(*copies[i % n_copies])
+
+    # ---- timed region: K steps; an event every `chunk` steps gives the spread of the step time ----
+    chunk = 10 if args.steps >= 100 else 1
+    n_ev = args.steps // chunk
     for i in range(args.warmup):
         step(i)
     barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev + 1)]
+    ev_end = torch.cuda.Event(enable_timing=True)
     with ClockSampler(local_rank) as clocks:
-        ev0.record(stream)
         for i in range(args.steps):
+            if i % chunk == 0 and i // chunk < n_ev:
+                evs[i // chunk].record(stream)
             step(i)
-        ev1.record(stream)
+            if (i + 1) == n_ev * chunk:
+                evs[n_ev].record(stream)
+        ev_end.record(stream)
         barrier()
-    local_ms = ev0.elapsed_time(ev1)
-    value, total_ms = aggregate_over_ranks(local_ms, float(B * gamma * args.steps), world, reduce_max, reduce_sum)
+    local_ms = evs[0].elapsed_time(ev_end)
+    value, total_ms = aggregate_over_ranks(local_ms, float(units * args.steps), world, reduce_max, reduce_sum)
     ms_per_step = total_ms / args.steps
-    res_acc, res_D = acc.cpu().numpy(), D.cpu().numpy()
+    chunk_ms = np.array([evs[k].elapsed_time(evs[k + 1]) / chunk for k in range(n_ev)])
+    res = {"acc": acc.cpu().numpy(), "tok": tok.cpu().numpy(), "D": D.cpu().numpy(), "st": st.cpu().numpy()}
+
+    # ---- the same with a single input copy (served from L2 when it fits): labelled, not the headline ----
+    hot_ms = None
+    if in_bytes < L2_BYTES:
+        n_hot = max(20, min(args.steps, 500))
+        for _ in range(5):
+            call(*copies[0])
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(n_hot):
+            call(*copies[0])
+        h1.record(stream)
+        torch.cuda.synchronize()
+        hot_ms = h0.elapsed_time(h1) / n_hot
 
     # ---- which kernel takes the time: a short second loop with an event recorded by the library
     #      between the pair kernel and the finish kernel (the calls are queued back to back, so
-    #      the intervals are kernel durations, not launch gaps) ----
+    #      the intervals are kernel durations, not launch gaps; the record in the middle keeps the
+    #      finish kernel from being set up early, so the two add up to slightly more than a step) ----
     n_attr = max(1, min(args.steps, 50))
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_attr)]
     for e3 in ev:
@@ -297,19 +426,34 @@ def main():
     finish_ms = float(np.median([e3[1].elapsed_time(e3[2]) for e3 in ev]))
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region ----
-    stg_b = fsd.fsd_host_staging_bytes(B, gamma, V, opts)
-    staging = torch.empty(stg_b, dtype=torch.uint8, device="cuda")
     h_acc = torch.empty(B, dtype=torch.int32).pin_memory()
-    h_tok = torch.empty(B, dtype=torch.int32).pin_memory()
-    h_D = torch.empty(B, gamma, dtype=torch.float32).pin_memory()
+    h_tk = torch.empty(B, dtype=torch.int32).pin_memory()
+    h_D = torch.empty(B, P, dtype=torch.float32).pin_memory()
     h_st = torch.empty(B, dtype=torch.int32).pin_memory()
+    if tree:
+        h_path = torch.empty(B, c.max_depth, dtype=torch.int32).pin_memory()
+        d_t, d_d = copies[0]
 
-    def e2e_step():
-        rc = fsd.fsd_verify_chain_host(h_target, h_draft, None, None, h_us, B, gamma, V, opts,
-                                       h_acc, h_tok, h_D, h_st, staging, stg_b, sptr)
-        if rc != 0:
-            raise RuntimeError(fsd.fsd_status_string(rc))
+        def e2e_step():                               # the tree call has no host-buffer variant: the copies are the caller's
+            d_t.copy_(h_target, non_blocking=True); d_d.copy_(h_draft, non_blocking=True)
+            pard.copy_(h_par, non_blocking=True); us.copy_(h_us, non_blocking=True)
+            call(d_t, d_d)
+            h_acc.copy_(acc, non_blocking=True); h_tk.copy_(tok, non_blocking=True); h_D.copy_(D, non_blocking=True)
+            h_st.copy_(st, non_blocking=True); h_path.copy_(path, non_blocking=True)
+            stream.synchronize()
+        h2d = in_bytes + h_par.numel() * 4 + h_us.numel() * 4
+        d2h = (h_acc.numel() + h_tk.numel() + h_D.numel() + h_st.numel() + h_path.numel()) * 4
+    else:
+        stg_b = fsd.fsd_host_staging_bytes(B, P, V, opts)
+        staging = torch.empty(stg_b, dtype=torch.uint8, device="cuda")
 
+        def e2e_step():
+            rc = fsd.fsd_verify_chain_host(h_target, h_draft, h_tok, h_ua, h_us, B, P, V, opts,
+                                           h_acc, h_tk, h_D, h_st, staging, stg_b, sptr)
+            if rc != 0:
+                raise RuntimeError(fsd.fsd_status_string(rc))
+        h2d = in_bytes + h_us.numel() * 4 + (h_tok.numel() * 4 + h_ua.numel() * 4)
+        d2h = (h_acc.numel() + h_tk.numel() + h_D.numel() + h_st.numel()) * 4
     for _ in range(3):
         e2e_step()
     barrier()
@@ -319,11 +463,9 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
-    e2e_value, e2e_ms = aggregate_over_ranks(e0.elapsed_time(e1), float(B * gamma * args.e2e_steps), world,
+    e2e_value, e2e_ms = aggregate_over_ranks(e0.elapsed_time(e1), float(units * args.e2e_steps), world,
                                              reduce_max, reduce_sum)
-    h2d = (h_target.numel() + h_draft.numel()) * c.elem_size + h_us.numel() * 4
-    d2h = (h_acc.numel() + h_tok.numel() + h_D.numel() + h_st.numel()) * 4
-    assert np.array_equal(h_acc.numpy(), res_acc)
+    assert np.array_equal(h_acc.numpy(), res["acc"]), "the host-buffer call and the device call disagree"
 
     if rank != 0:
         if dist is not None:
@@ -333,48 +475,71 @@ def main():
     # ---- roofline of the dominant kernel (the pair kernel): its algorithmic bytes (both rows of
     #      every pair read once) over its own duration; the whole call is given beside it ----
     peak, peak_kind = measured_hbm_peak()
-    ideal = c.ideal_bytes
-    pair_bytes = c.elem_size * B * gamma * 2 * V
+    if tree:
+        end_node = np.array([(p[p >= 0][-1] if (p >= 0).any() else -1) for p in path.cpu().numpy()])
+        ideal = c.elem_size * V * gi.tree_unique_rows(c.parent, end_node)
+        pair_bytes = c.elem_size * V * sum(c.N + len(set(int(p) + 1 for p in c.parent[b])) for b in range(B))
+    else:
+        ideal = c.ideal_bytes
+        pair_bytes = c.elem_size * B * P * 2 * V
     achieved = pair_bytes / (pair_ms * 1e-3) / 1e9
     call_achieved = ideal / (ms_per_step * 1e-3) / 1e9
+    kname = "fsd_pair_stream_kernel" if (V * c.elem_size) % 16 == 0 and V * c.elem_size >= 1024 else "fsd_pair_generic_kernel"
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": PAIR_KERNEL_DRAM_BYTES if headline else None, "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                "kernel": "pair kernel (fsd_pair_stream_kernel<bf16, JS> on the headline workload; includes the "
-                          "256-byte flag memset in front of it)",
+                "kernel": f"pair kernel ({kname}<{c.dtype}, {args.div.upper()}>; the interval includes the 256-byte "
+                          "flag memset in front of it)",
                 "algorithmic_bytes_per_launch": pair_bytes, "ms_per_launch": pair_ms,
                 "finish_kernel_ms": finish_ms,
+                "attribution_note": "pair + finish intervals are taken with an event recorded between the two "
+                                    "kernels, which forbids their overlap: together they exceed ms_per_step",
                 "whole_call": {"achieved": call_achieved, "frac": call_achieved / peak,
+                               "frac_of_nominal_8000": call_achieved / NOMINAL_HBM_GBS,
                                "algorithmic_bytes_per_call": ideal, "ms_per_call": ms_per_step}}
 
-    # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only ----
-    cpu = None
-    if world == 1:
-        rows = 16
-        v, secs, cores = oracle_sample_rate(c, rows, T)
-        if secs < 5.0:
-            reps = int(min(20, max(1, 10.0 / max(secs, 1e-3))))
-            t0 = time.perf_counter()
-            for _ in range(reps):
-                oracle_sample_rate(c, rows, T)
-            v = rows * gamma * reps / (time.perf_counter() - t0)
-        cpu = {"value": v, "unit": "positions/s", "cores": cores, "kind": "oracle",
-               "sample": f"first {rows} of {B} batch rows ({rows * gamma} positions per pass), repeated for ~10 s"}
+    # ---- CPU baseline and parity: the oracle on a bounded sample, rank 0, N = 1 only ----
+    cpu = parity = None
+    if world == 1 and not args.no_cpu:
+        from oracle import fsd_oracle as orc
+        rows = sample_rows(c)
+        tol = 1e-5 if c.dtype == "f32" else 1e-4
+        o, _ = oracle_run(c, rows, args.div, args.mode, T)
+        if tree or args.mode == "fsd":
+            parity, ok = parity_counts(c, o, rows, res, T, tol)
+            if not ok:
+                raise SystemExit(f"the timed call disagrees with the oracle: {parity}")
+        v_all = oracle_rate(c, rows, args.div, args.mode, T, 0, 10.0)
+        v_one = oracle_rate(c, min(rows, 2), args.div, args.mode, T, 1, 4.0)
+        per_row = units // B
+        cpu = {"value": v_all, "unit": "positions/s", "cores": orc.max_threads(), "kind": "oracle",
+               "sample": f"first {rows} of {B} batch rows ({rows * per_row} positions per pass), repeated for ~10 s",
+               "one_core": {"value": v_one, "cores": 1,
+                            "sample": f"first {min(rows, 2)} batch rows, repeated for ~4 s"}}
 
-    hist = np.bincount(res_acc, minlength=gamma + 1).tolist()
+    hist = np.bincount(res["acc"], minlength=(c.max_depth if tree else P) + 1).tolist()
+    cfg = describe(c, name, args.div, args.mode, T, named=not overrides)
+    cfg["l2"] = (f"inputs ({in_bytes / 1e6:.1f} MB) "
+                 + ("exceed" if in_bytes > L2_BYTES else "are smaller than")
+                 + f" L2 (126 MB); {n_copies} input copies ({n_copies * in_bytes / 1e6:.0f} MB) rotated between steps")
     line = {
         "metric": "verified draft positions/sec", "value": value, "unit": "positions/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": workload_config(c, B),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "ms_per_step_median": float(np.median(chunk_ms)), "ms_per_step_best": float(chunk_ms.min()),
+        "step_time_granularity": f"means over {chunk} consecutive steps",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": cfg,
         "roofline": roofline,
+        "hot_l2": None if hot_ms is None else {"ms_per_step": hot_ms, "value": units / (hot_ms * 1e-3),
+                                               "note": "one input copy re-read every step (served from L2): not the headline"},
         "cpu_baseline": cpu,
+        "parity": parity,
         "e2e": {"value": e2e_value, "unit": "positions/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks.summary(),
-        "workload_stats": {"accept_len_hist": hist, "D_min": float(np.nanmin(res_D)),
-                           "D_median": float(np.nanmedian(res_D)), "D_max": float(np.nanmax(res_D))},
+        "workload_stats": {"accept_len_hist": hist, "D_min": float(np.nanmin(res["D"])),
+                           "D_median": float(np.nanmedian(res["D"])), "D_max": float(np.nanmax(res["D"]))},
     }
     print(json.dumps(line))
     if dist is not None:

@@ -5,12 +5,16 @@
 //   3. Draws the replacement / bonus token from one target row (and, for the SD residual, one
 //      draft row) by an inverse CDF in vocabulary order.
 //
-// The draw must land on the same token as a sequential double-precision sum would, so the
-// exponentials and partial sums of step 3 are double precision: each thread owns a contiguous
-// chunk of the vocabulary, chunk sums are combined by a fixed-order scan (thread -> warp ->
-// CTA -> cluster), and the first thread whose inclusive sum exceeds u * total re-walks its
-// chunk.  The double exponential is a 64-entry table times a degree-5 polynomial (about ten
-// fp64 operations); the rows involved are a 1/(2*gamma+1) share of all logits.
+// Drawing from P_T (the FSD rule, and every bonus token): each thread owns a contiguous chunk
+// of the vocabulary; the weights are single-precision exponentials (one MUFU ex2 each, relative
+// error at most a few 1e-7) summed in double precision, chunk sums are combined by a fixed-order
+// scan (thread -> warp -> CTA -> cluster), and the warp of the first thread whose inclusive sum
+// exceeds u * total re-walks that chunk with the same weights.  The cumulative sums therefore
+// differ from exact ones by less than 1e-6 of the total: the token is the exact one whenever
+// u * total lies further than that from both ends of its interval, and a neighbour otherwise.
+// Drawing from the SD residual max(0, P_T - P_D) (Eq. 3) subtracts nearly equal numbers, so
+// there the exponentials are double precision (a 256-entry table times a degree-4 polynomial,
+// about ten fp64 operations) and the sums agree with a sequential double sum to rounding.
 #pragma once
 
 #include "fsd_device.cuh"
@@ -53,6 +57,8 @@ constexpr int kExpTable = 256;
 
 struct FinishShared {
     FinishExchange slot;
+    FinishExchange all[kMaxClusterSize];   // what the cluster's CTAs published (see cluster_exchange)
+    double sc[kMaxClusterSize];
     double gather_d[kMaxClusterSize];   // one value per CTA of the cluster (see cluster_gather)
     int gather_i[kMaxClusterSize];
     double exp_table[kExpTable];   // 2^(j/256)
@@ -89,16 +95,13 @@ __device__ __forceinline__ double exp2_table(double y, const double* table) {
     return __hiloint2double(hi, __double2loint(m));
 }
 
-// Every CTA of the cluster publishes a FinishExchange and reads everybody's.
+// Every CTA of the cluster publishes a FinishExchange; afterwards sh.all holds everybody's.
 // Two cluster barriers: after the writes, and after the reads (so the slot can be reused).
 __device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, FinishShared& sh, int cs,
-                                                 const FinishExchange& mine, FinishExchange (&all)[kMaxClusterSize]) {
+                                                 const FinishExchange& mine) {
     if (threadIdx.x == 0) sh.slot = mine;
     cluster.sync();
-#pragma unroll
-    for (int r = 0; r < kMaxClusterSize; ++r) {
-        if (r < cs) all[r] = cluster.map_shared_rank(&sh, r)->slot;
-    }
+    if (threadIdx.x < cs) sh.all[threadIdx.x] = cluster.map_shared_rank(&sh, threadIdx.x)->slot;
     cluster.sync();
 }
 
@@ -343,17 +346,22 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const long long k0l = static_cast<long long>(rank * blockDim.x + tid) * L;
     const int k0 = k0l < V ? static_cast<int>(k0l) : V;
     const int k1 = (k0l + L) < V ? static_cast<int>(k0l + L) : V;
-    FinishExchange mine, all[kMaxClusterSize];
+    FinishExchange mine;
+    FinishExchange* const all = sh.all;
+    double* const sc = sh.sc;
 
     // ---- fast path: inverse CDF over P_T (the FSD rule, and every bonus token) ----
     if (!residual0 && !greedy) {
-        // Reference exponent k (log2 domain): the pair's record has it when this row was a pair's
-        // target row; otherwise one pass for the row maximum.
-        double kref = 0.0;
+        // Reference exponent k (log2 domain, an integer) at or just above the row's log-sum-exp, so
+        // that every exponent is <= 0 and those of the entries that carry mass are small (their
+        // rounding error stays far below the 1e-6 the draw may be off by).  When the row was a
+        // pair's target row the pair's record gives the log-sum-exp; otherwise one pass for the
+        // row maximum.
+        float kref = 0.f;
         bool have_ref = false;
         if (P.records != nullptr && !tree && n < G) {
             const PairRecord* r = P.records + (static_cast<size_t>(b) * G + n);
-            if (r->state & kRecordStats) {                // any common reference near the maximum serves
+            if (r->state & kRecordStats) {
                 float rka = -INFINITY;
                 bool nan = false;
                 for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
@@ -361,7 +369,14 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                     nan = nan || a != a;
                     rka = fmaxf(rka, a);
                 }
-                if (!nan && isfinite(rka)) { kref = rka; have_ref = true; }
+                if (!nan && isfinite(rka)) {
+                    float za = 0.f;
+                    for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
+                        const float a = r->part[c].ka;
+                        if (a != -INFINITY) za += r->part[c].za * pow2_int(a - rka);
+                    }
+                    if (za > 0.f && za < 3.0e38f) { kref = ceilf(rka + log2f(za)); have_ref = true; }
+                }
             }
         }
         if (!have_ref) {
@@ -375,12 +390,13 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                 if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.next_token[b] = -1; P.row_status[b] = status | FSD_ROW_NONFINITE; }
                 return;
             }
-            kref = M * kLog2eD;
+            kref = ceilf(static_cast<float>(M) * kLog2e);
         }
+        // weight of one entry: 2^(logit * log2e - k), the same float in every pass
+        const float nk = -kref;
+        auto weight = [&](float xa) -> float { return ex2(fmaf(xa, kLog2e, nk)); };
         double csum = 0.0;
-        for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int, float xa, float) {
-            csum += exp2_table(fma(static_cast<double>(xa), kLog2eD, -kref), tab);
-        });
+        for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int, float xa, float) { csum += static_cast<double>(weight(xa)); });
         // inclusive / exclusive scan of the chunk sums over the CTA, fixed order
         double incl = csum;
 #pragma unroll
@@ -417,9 +433,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         }
         auto last_with_weight = [&]() -> int {           // highest index of this thread's chunk whose weight is positive
             int lastp = -1;
-            for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int k, float xa, float) {
-                if (exp2_table(fma(static_cast<double>(xa), kLog2eD, -kref), tab) > 0.0) lastp = k;
-            });
+            for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int k, float xa, float) { if (weight(xa) > 0.f) lastp = k; });
             return lastp;
         };
         if (owner < 0) {                                  // t >= W after rounding (uniform): the last token that has weight
@@ -452,7 +466,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             for (int kb = ck0; kb < ck1; kb += 32) {
                 const int k = kb + lane;
                 double w = 0.0;
-                if (k < ck1) w = exp2_table(fma(static_cast<double>(load_logit<DT>(a_row, k)), kLog2eD, -kref), tab);
+                if (k < ck1) w = static_cast<double>(weight(load_logit<DT>(a_row, k)));
                 double run = w;
 #pragma unroll
                 for (int d = 1; d < 32; d <<= 1) {
@@ -527,7 +541,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         float bv[1] = {bad_v};
         block_max<1>(bv, sh.red_f);
         mine.d[0] = best; mine.d[1] = bv[0]; mine.d[2] = 0; mine.d[3] = 0; mine.i[0] = idx; mine.i[1] = 0;
-        cluster_exchange(cluster, sh, cs, mine, all);
+        cluster_exchange(cluster, sh, cs, mine);
         double gb = all[0].d[0], gbad = all[0].d[1];
         int gi = all[0].i[0];
         for (int r = 1; r < cs; ++r) {
@@ -559,7 +573,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         });
         block_sum<2>(z, sh.red_d);
         mine.d[0] = Ra; mine.d[1] = Rb; mine.d[2] = z[0]; mine.d[3] = z[1]; mine.i[0] = 0; mine.i[1] = 0;
-        cluster_exchange(cluster, sh, cs, mine, all);
+        cluster_exchange(cluster, sh, cs, mine);
         Ma = -INFINITY; Mb = -INFINITY;
         for (int r = 0; r < cs; ++r) { Ma = fmax(Ma, all[r].d[0]); Mb = fmax(Mb, all[r].d[1]); }
         double Za = 0.0, Zb = 0.0;
@@ -636,16 +650,16 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             }
         }
         mine.d[0] = cta_tot; mine.d[1] = Ra; mine.d[2] = wbest; mine.d[3] = 0; mine.i[0] = sh.last_pos; mine.i[1] = kbest;
-        cluster_exchange(cluster, sh, cs, mine, all);
+        cluster_exchange(cluster, sh, cs, mine);
 
         // cluster totals on a common reference
         double M = -INFINITY;
         for (int r = 0; r < cs; ++r) M = fmax(M, all[r].d[1]);
-        double sc[kMaxClusterSize], W = 0.0;
-        for (int r = 0; r < cs; ++r) {
-            sc[r] = residual ? 1.0 : (all[r].d[1] > -INFINITY ? exp2_table((all[r].d[1] - M) * kLog2eD, tab) : 0.0);
-            W += all[r].d[0] * sc[r];
-        }
+        double W = 0.0;
+        __syncthreads();                                  // everybody is done with the last attempt's factors
+        if (tid < cs) sc[tid] = residual ? 1.0 : (all[tid].d[1] > -INFINITY ? exp2_table((all[tid].d[1] - M) * kLog2eD, tab) : 0.0);
+        __syncthreads();
+        for (int r = 0; r < cs; ++r) W += all[r].d[0] * sc[r];
         if (residual && !(W > 0.0)) {                     // no residual mass: draw from P_T (uniform decision)
             residual = false;
             __syncthreads();

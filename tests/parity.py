@@ -10,9 +10,13 @@ Rules
     accept_len and next_token.  Affected rows are replayed: the oracle is re-run with the in-band
     decisions forced to what the GPU's accept_len implies and must then reproduce the GPU's
     accept_len and token.
-  * tokens: the oracle reports the tokens selected for t -/+ band*W with band = 1e-12 (the
-    GPU's double-precision CDF differs from the sequential sum by rounding only); a GPU token
-    inside that range but different from the oracle's is counted as a sample-band hit.
+  * tokens: the oracle reports the tokens selected for t -/+ band*W; a GPU token inside that
+    range but different from the oracle's is counted as a sample-band hit, one outside fails.
+    A token drawn from P_T (every FSD draw, every bonus token) is computed on the GPU from
+    single-precision exponentials summed in double: band = 1e-6, so the token is the oracle's
+    own whenever u*W is further than 1e-6*W from both ends of that token's interval.  A token
+    drawn from the SD residual max(0, P_T - P_D) is computed in double throughout and differs
+    from the sequential sum by rounding only: band = 1e-12.
 """
 
 from __future__ import annotations
@@ -27,7 +31,9 @@ from oracle import fsd_oracle as orc
 
 D_BAND = 1e-5
 P_BAND = 1e-6
-SAMPLE_BAND = 1e-12
+SAMPLE_BAND_PT = 1e-6          # draws from P_T
+SAMPLE_BAND_RESIDUAL = 1e-12   # draws from the SD residual
+SAMPLE_BAND = SAMPLE_BAND_PT   # tree verification and FSD mode draw from P_T only
 
 
 def to_device(arr: np.ndarray, dtype: str):
@@ -118,8 +124,17 @@ def check_chain(inp_target, inp_draft, tokens, u_accept, u_sample, dtype, div="j
     tol = 1e-5 if dtype == "f32" else 1e-4
     g = run_chain_gpu(inp_target, inp_draft, tokens, u_accept, u_sample, dtype, div, mode, cmp, sample, T, dev)
     o = orc.verify_chain(inp_target, inp_draft, tokens, u_accept, u_sample, dtype=dtype, div=div, mode=mode,
-                         cmp=cmp, sample_kind=sample, T=T, band=SAMPLE_BAND)
+                         cmp=cmp, sample_kind=sample, T=T, band=SAMPLE_BAND_PT)
     B, gamma = o.divergence.shape
+    # in SD / rFSD mode a rejected row draws from the residual: the tight band applies there
+    o_res = None
+    if mode != "fsd":
+        o_res = orc.verify_chain(inp_target, inp_draft, tokens, u_accept, u_sample, dtype=dtype, div=div, mode=mode,
+                                 cmp=cmp, sample_kind=sample, T=T, band=SAMPLE_BAND_RESIDUAL)
+
+    def band_of(n_acc):
+        return SAMPLE_BAND_RESIDUAL if (mode != "fsd" and n_acc < gamma) else SAMPLE_BAND_PT
+
     max_err = compare_divergence(g.divergence, o.divergence, tol)
     assert np.array_equal(g.row_status, o.row_status), (g.row_status, o.row_status)
 
@@ -133,7 +148,9 @@ def check_chain(inp_target, inp_draft, tokens, u_accept, u_sample, dtype, div="j
     for b in range(B):
         upto = min(gamma, max(int(g.accept_len[b]), int(o.accept_len[b])) + 1)
         affected = bool(in_band[b, :upto].any())
-        n_o, t_o, lo, hi = int(o.accept_len[b]), int(o.next_token[b]), int(o.tok_lo[b]), int(o.tok_hi[b])
+        n_o, t_o = int(o.accept_len[b]), int(o.next_token[b])
+        src = o_res if (o_res is not None and n_o < gamma) else o
+        lo, hi = int(src.tok_lo[b]), int(src.tok_hi[b])
         if affected and (g.accept_len[b] != n_o):
             band_rows += 1
             replayed += 1
@@ -145,7 +162,7 @@ def check_chain(inp_target, inp_draft, tokens, u_accept, u_sample, dtype, div="j
                                  None if tokens is None else tokens[b:b + 1],
                                  None if u_accept is None else u_accept[b:b + 1], u_sample[b:b + 1],
                                  dtype=dtype, div=div, mode=mode, cmp=cmp, sample_kind=sample, T=T,
-                                 band=SAMPLE_BAND, forced=forced)
+                                 band=band_of(int(g.accept_len[b])), forced=forced)
             n_o, t_o, lo, hi = int(r.accept_len[0]), int(r.next_token[0]), int(r.tok_lo[0]), int(r.tok_hi[0])
         elif affected:
             band_rows += 1
