@@ -4,15 +4,15 @@
  *
  * What a call computes, for every batch row b and candidate position i:
  *   1. P_T[i] = softmax(target_logits[b, i, :]), P_D[i] = softmax(draft_logits[b, i, :])
- *      (Section 4: "next token distributions at candidate position i").
+ *      (Section 4, the two distributions compared by Eq. 4).
  *   2. The divergence D[b, i] = Div(P_T[i], P_D[i]) in nats: Jensen-Shannon
  *      (Appendix C.2, the paper's default), KL(P_T || P_D) (Appendix C.1) or total
  *      variation (Appendix C.3).
  *   3. The acceptance bit: FSD accepts iff D < T (Section 4, Eq. 4; "<=" selectable);
  *      SD accepts iff u_accept < min(1, P_T(x_i)/P_D(x_i)) (Section 3, Eq. 1-2);
  *      rFSD accepts iff either holds (Section 4.3, Eq. 6).
- *   4. accept_len[b] = index of the first rejected position, or gamma (Section 3,
- *      "first rejection").
+ *   4. accept_len[b] = index of the first rejected position, or gamma (Section 3: the
+ *      candidates before the earliest failing test are kept).
  *   5. next_token[b]: FSD draws it from P_T at the rejected position (Section 4);
  *      SD and rFSD from max(0, P_T - P_D) renormalised (Section 3, Eq. 3); when every
  *      candidate was accepted it is drawn from P_T of the extra row gamma.  The draw
@@ -32,7 +32,9 @@
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
  *     default stream).  Outputs are valid once the stream has been synchronised.
  *   - The return value is a host-side status: FSD_OK (0) or a negative FSD_ERR_*.
- *     On error nothing has been launched.  Nothing aborts, throws or traps.
+ *     On error no kernel of the call has run (a launch the runtime refuses, FSD_ERR_CUDA, can
+ *     leave a 256-byte memset of the workspace's flag block on the stream; everything that
+ *     can fail before that is checked first).  Nothing aborts, throws or traps.
  *   - Conditions found on the device are reported per batch row in row_status.
  *   - -inf logits are legal (probability zero).  A row holding NaN, +inf or no finite
  *     value makes its position's divergence NaN, rejects the position and sets
@@ -174,6 +176,8 @@ int fsd_verify_chain_host(const void *h_target_logits, const void *h_draft_logit
  *     is resident on every GPU that loads the library until the process exits.
  *   - The first call on each device looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.
+ *     The address is remembered for the life of the process: do not reset the device
+ *     (cudaDeviceReset) between calls; after a reset the remembered address is stale.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.
  *     Nothing in it has to start at zero: every word a call reads was written earlier by the
  *     same call.  Two calls that overlap on the GPU (different streams, no ordering between
@@ -203,6 +207,14 @@ int fsd_version(void);
  * kernels also keeps the finish kernel from being set up early, so timings taken with the hook
  * are for attribution, not throughput.  Returns FSD_OK. */
 int fsd_set_stage_event(void *event);
+
+/* Test aid (no counterpart in the paper).  Every wait inside the streaming kernel is bounded; a
+ * wait that runs out raises a flag in the workspace, the call still returns, and every row's
+ * row_status carries FSD_ROW_TIMEOUT (its other outputs are then not valid).  While injection is
+ * on, verify calls raise that flag themselves (a 4-byte memset between the two kernels), so the
+ * reporting path can be exercised without making a GPU wait for something that never comes.
+ * Process-wide, read when a call is made; off by default.  Returns FSD_OK. */
+int fsd_set_timeout_injection(int on);
 
 /* ---- Threshold tuning (Section "Selecting T"; Discussion, "Potential further developments") ----
  * The paper tunes T on a small development set by running FSD at candidate thresholds and

@@ -85,6 +85,8 @@ def _load():
         lib.fsd_version.restype = C.c_int
         lib.fsd_set_stage_event.argtypes = [C.c_void_p]
         lib.fsd_set_stage_event.restype = C.c_int
+        lib.fsd_set_timeout_injection.argtypes = [C.c_int]
+        lib.fsd_set_timeout_injection.restype = C.c_int
         lib.fsd_threshold_sweep.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, C.c_int, vp, vp, C.c_void_p]
         lib.fsd_threshold_sweep.restype = C.c_int
         lib.fsd_calibrate_threshold.argtypes = [vp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, C.c_void_p]
@@ -132,6 +134,12 @@ def fsd_set_stage_event(event) -> int:
     if event is not None:
         handle = getattr(event, "cuda_event", event)
     return _load().fsd_set_stage_event(handle)
+
+
+def fsd_set_timeout_injection(on: bool) -> int:
+    """While on, verify calls report FSD_ROW_TIMEOUT in every row as if a bounded device-side wait
+    had run out (a test aid; off by default)."""
+    return _load().fsd_set_timeout_injection(1 if on else 0)
 
 
 def fsd_workspace_bytes(B: int, positions: int, V: int, opts: FsdOpts) -> int:

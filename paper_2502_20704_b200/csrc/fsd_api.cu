@@ -74,12 +74,28 @@ int finish_cluster_size(int B, int V) {
 }
 
 std::atomic<void*> g_stage_event{nullptr};   // see fsd_set_stage_event
+std::atomic<int> g_mark_timeout{0};          // see fsd_set_timeout_injection
 
 // ---- streaming kernel launch -----------------------------------------------------------
 constexpr int kMaxDev = 64;
 
+inline void stream_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int C, cudaStream_t s) {
+    cfg = {};
+    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.dynamicSmemBytes = kStreamSmemBytes;
+    cfg.stream = s;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+}
+
+// Attributes of the kernel and the number of clusters that can be resident (cached per device and
+// cluster size).  Puts nothing on a stream.
 template <int DT, int DIV>
-int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
+int prepare_stream(int C, int* nclus_out) {
     static int max_clusters[kMaxDev][5] = {};       // per device, per log2(C); 0 = not yet queried
     static std::mutex mu;
     auto kernel = fsd_pair_stream_kernel<DT, DIV>;
@@ -87,44 +103,40 @@ int launch_stream(const StreamParams& sp, int C, cudaStream_t s) {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return FSD_ERR_CUDA;
     int lc = 0;
     while ((1 << lc) < C) ++lc;
-
-    cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(kStreamThreads, 1, 1);
-    cfg.dynamicSmemBytes = kStreamSmemBytes;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = C;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    int nclus;
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        if (max_clusters[dev][lc] == 0) {
-            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+    std::lock_guard<std::mutex> lock(mu);
+    if (max_clusters[dev][lc] == 0) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+            return FSD_ERR_CUDA;
+        if (cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+            return FSD_ERR_CUDA;
+        if (C > 8) {                            // above the portable cluster size: opt in
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+                cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
                 return FSD_ERR_CUDA;
-            if (cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
-                return FSD_ERR_CUDA;
-            if (C > 8) {                            // above the portable cluster size: opt in
-                if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-                    cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
-                    return FSD_ERR_CUDA;
-            }
-            cfg.gridDim = dim3(C, 1, 1);
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, fsd_stream_occupancy_twin, &cfg) != cudaSuccess || n < 1)
-                return FSD_ERR_CUDA;
-            max_clusters[dev][lc] = n;
         }
-        nclus = max_clusters[dev][lc];
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[1];
+        stream_config(cfg, attr, C, nullptr);
+        cfg.gridDim = dim3(C, 1, 1);
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, fsd_stream_occupancy_twin, &cfg) != cudaSuccess || n < 1)
+            return FSD_ERR_CUDA;
+        max_clusters[dev][lc] = n;
     }
+    *nclus_out = max_clusters[dev][lc];
+    return FSD_OK;
+}
+
+template <int DT, int DIV>
+int launch_stream(const StreamParams& sp, int C, int nclus, cudaStream_t s) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    stream_config(cfg, attr, C, s);
     if (nclus > sp.n_items) nclus = sp.n_items;
     cfg.gridDim = dim3(static_cast<unsigned>(nclus) * C, 1, 1);
-    if (cudaLaunchKernelEx(&cfg, kernel, sp) != cudaSuccess) return FSD_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, fsd_pair_stream_kernel<DT, DIV>, sp) != cudaSuccess) return FSD_ERR_CUDA;
     return FSD_OK;
 }
 
@@ -146,13 +158,21 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Pair
         StreamParams sp;
         sp.target = pp.target; sp.draft = pp.draft; sp.parent = pp.parent; sp.B = pp.B; sp.G = pp.G;
         sp.nvec_row = nvec_row; sp.n_items = items; sp.records = records; sp.timeout_flag = flags; sp.next_pair = flags + 1;
+        // everything that can fail without a launch (attributes, the occupancy query) comes before
+        // the first thing put on the stream
+        int rc, nclus = 0;
+        if (pp.div == FSD_DIV_JS)      rc = prepare_stream<DT, FSD_DIV_JS>(C, &nclus);
+        else if (pp.div == FSD_DIV_KL) rc = prepare_stream<DT, FSD_DIV_KL>(C, &nclus);
+        else                           rc = prepare_stream<DT, FSD_DIV_TV>(C, &nclus);
+        if (rc != FSD_OK) return rc;
         // the flag block starts every call at zero: [0] timeout, [1] pairs handed out
         if (cudaMemsetAsync(flags, 0, kAlign, s) != cudaSuccess) return FSD_ERR_CUDA;
-        int rc;
-        if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, C, s);
-        else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, C, s);
-        else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, C, s);
+        if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, C, nclus, s);
+        else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, C, nclus, s);
+        else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, C, nclus, s);
         if (rc != FSD_OK) return rc;
+        // test aid: behave as if a bounded wait of the streaming kernel had run out
+        if (g_mark_timeout.load() != 0 && cudaMemsetAsync(flags, 1, sizeof(int), s) != cudaSuccess) return FSD_ERR_CUDA;
         fp.timeout_flag = flags;
         fp.records = records;
     } else {
@@ -422,11 +442,17 @@ int fsd_set_stage_event(void* event) {
     return FSD_OK;
 }
 
+int fsd_set_timeout_injection(int on) {
+    g_mark_timeout.store(on != 0 ? 1 : 0);
+    return FSD_OK;
+}
+
 int fsd_threshold_sweep(const float* divergence, int B, int positions, const float* thresholds, int n_thresholds,
                         int compare, float* mean_accept_len, float* accept_fraction, void* stream) {
     if (divergence == nullptr || thresholds == nullptr || mean_accept_len == nullptr || accept_fraction == nullptr)
         return FSD_ERR_NULL;
     if (B < 1 || positions < 1 || n_thresholds < 1) return FSD_ERR_SHAPE;
+    if (static_cast<long long>(B) * positions > INT_MAX) return FSD_ERR_SHAPE;      // the kernels count in 32 bits
     if (compare != FSD_CMP_LT && compare != FSD_CMP_LE) return FSD_ERR_ENUM;
     fsd_threshold_sweep_kernel<<<n_thresholds, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         divergence, B, positions, thresholds, compare, mean_accept_len, accept_fraction);
@@ -437,6 +463,7 @@ int fsd_calibrate_threshold(const float* divergence, int B, int positions, float
                             float* threshold_out, float* achieved_out, void* stream) {
     if (divergence == nullptr || threshold_out == nullptr || achieved_out == nullptr) return FSD_ERR_NULL;
     if (B < 1 || positions < 1 || !(target_mean_accept_len >= 0.f)) return FSD_ERR_SHAPE;   // NaN target included
+    if (static_cast<long long>(B) * positions > INT_MAX) return FSD_ERR_SHAPE;      // the kernels count in 32 bits
     if (compare != FSD_CMP_LT && compare != FSD_CMP_LE) return FSD_ERR_ENUM;
     fsd_calibrate_kernel<<<1, kTuneThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         divergence, B, positions, target_mean_accept_len, compare, threshold_out, achieved_out);

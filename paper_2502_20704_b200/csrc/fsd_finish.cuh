@@ -71,6 +71,8 @@ struct FinishShared {
     int row_sel;               // target row the token is drawn from
     int n_acc;
     int bad;
+    int best_key;              // depth * 2048 + (2047 - node) of the chosen tree node, or -1
+    int16_t tree_jump[kMaxTreeNodes];
     int16_t tree_depth[kMaxTreeNodes];
     int8_t tree_ok[kMaxTreeNodes];
     int8_t tree_bit[kMaxTreeNodes];
@@ -236,6 +238,73 @@ __device__ __forceinline__ void for_chunk(const void* a_row, const void* b_row, 
     }
 }
 
+// Tree: the deepest node whose whole path passes (ties: lowest index), its depth and path.
+// Called by all threads of the CTA; leaves sh.n_acc / sh.row_sel and writes the path if `pth` is given.
+__device__ __noinline__ void tree_select(const int32_t* par, int G, int max_depth, int32_t* pth, FinishShared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    // Depth of every node and "all nodes from the root down to it pass", by pointer jumping:
+    // every node keeps (nodes counted, all pass, next ancestor) for the stretch of its path it
+    // has seen so far and doubles that stretch each round, so ceil(log2 N) rounds do for any
+    // tree shape (a serial walk takes N dependent steps for a chain-shaped tree of N nodes).
+    const bool good = !(sh.bad & FSD_ROW_BADTREE);
+    constexpr int kPer = (kMaxTreeNodes + kFinishThreads - 1) / kFinishThreads;
+    if (tid == 0) sh.best_key = -1;
+    if (good) {
+        for (int j = tid; j < G; j += kFinishThreads) {
+            sh.tree_jump[j] = static_cast<int16_t>(par[j]);
+            sh.tree_depth[j] = 1;
+            sh.tree_ok[j] = sh.tree_bit[j];
+        }
+        __syncthreads();
+        for (int span = 1; span < G; span <<= 1) {
+            int nj[kPer], nd[kPer], no[kPer];
+#pragma unroll
+            for (int q = 0; q < kPer; ++q) {
+                const int j = tid + q * kFinishThreads;
+                nj[q] = -1; nd[q] = 0; no[q] = 0;
+                if (j < G) {
+                    const int p = sh.tree_jump[j];
+                    nj[q] = p; nd[q] = sh.tree_depth[j]; no[q] = sh.tree_ok[j];
+                    if (p >= 0) { nj[q] = sh.tree_jump[p]; nd[q] += sh.tree_depth[p]; no[q] &= sh.tree_ok[p]; }
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int q = 0; q < kPer; ++q) {
+                const int j = tid + q * kFinishThreads;
+                if (j < G) {
+                    sh.tree_jump[j] = static_cast<int16_t>(nj[q]);
+                    sh.tree_depth[j] = static_cast<int16_t>(nd[q]);
+                    sh.tree_ok[j] = static_cast<int8_t>(no[q]);
+                }
+            }
+            __syncthreads();
+        }
+        // deepest passing node within max_depth, ties to the lowest index
+        int key = -1;
+        for (int j = tid; j < G; j += kFinishThreads) {
+            const int d = sh.tree_depth[j];
+            if (sh.tree_ok[j] && d <= max_depth) {
+                const int k = d * 2048 + (2047 - j);
+                key = k > key ? k : key;
+            }
+        }
+        key = __reduce_max_sync(0xffffffffu, key);
+        if (lane == 0 && key >= 0) atomicMax(&sh.best_key, key);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const int key = sh.best_key;
+        const int best = key < 0 ? -1 : 2047 - (key & 2047), best_depth = key < 0 ? 0 : key >> 11;
+        sh.n_acc = best_depth;
+        sh.row_sel = best + 1;
+        if (pth != nullptr) {
+            for (int d = 0; d < max_depth; ++d) pth[d] = -1;
+            for (int j = best, d = best_depth - 1; j >= 0 && d >= 0; j = par[j], --d) pth[d] = j;
+        }
+    }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishParams P) {
     __shared__ FinishShared sh;
@@ -298,30 +367,11 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     __syncthreads();
 
     // ---- 2. accepted prefix (chain) or deepest accepted path (tree) ----
-    if (tid == 0) {
-        if (!tree) {
-            sh.row_sel = sh.n_acc;
-        } else {
-            const int32_t* par = P.parent + static_cast<size_t>(b) * G;
-            int best = -1, best_depth = 0;
-            if (!(sh.bad & FSD_ROW_BADTREE)) {
-                for (int j = 0; j < G; ++j) {
-                    const int p = par[j];
-                    const int d = p < 0 ? 1 : sh.tree_depth[p] + 1;
-                    const bool ok = sh.tree_bit[j] && (p < 0 || sh.tree_ok[p]);
-                    sh.tree_depth[j] = static_cast<int16_t>(d);
-                    sh.tree_ok[j] = ok;
-                    if (ok && d <= P.max_depth && d > best_depth) { best = j; best_depth = d; }
-                }
-            }
-            sh.n_acc = best_depth;
-            sh.row_sel = best + 1;
-            if (rank == 0) {
-                int32_t* pth = P.path + static_cast<size_t>(b) * P.max_depth;
-                for (int d = 0; d < P.max_depth; ++d) pth[d] = -1;
-                for (int j = best, d = best_depth - 1; j >= 0; j = par[j], --d) pth[d] = j;
-            }
-        }
+    if (!tree) {
+        if (tid == 0) sh.row_sel = sh.n_acc;
+    } else {
+        tree_select(P.parent + static_cast<size_t>(b) * G, G, P.max_depth,
+                    rank == 0 ? P.path + static_cast<size_t>(b) * P.max_depth : nullptr, sh);
     }
     __syncthreads();
     const int n = sh.n_acc, row_sel = sh.row_sel;

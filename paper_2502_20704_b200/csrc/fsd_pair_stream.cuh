@@ -115,8 +115,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* timeout_flag, bool& dead) {
     if (dead) return false;
 #pragma unroll 1
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        // somebody has given up already: nothing this thread waits for is certain to come
+        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int*>(timeout_flag) != 0) break;
+    }
     atomicExch(timeout_flag, 1);
     dead = true;
     return false;
@@ -283,8 +286,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, int* timeout_flag, bool& dead) {
     if (dead) return false;
 #pragma unroll 1
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int*>(timeout_flag) != 0) break;
+    }
     atomicExch(timeout_flag, 1);
     dead = true;
     return false;
@@ -296,6 +301,7 @@ struct StreamShared {
     uint64_t xbar[2];          // all CTAs' statistics have landed here (per parity): 1 arrival + C * 32 bytes
     uint64_t empty[kRing];     // every warp has finished reading the slot's current stage
     uint32_t tmem_base;
+    uint32_t armed[kRing];     // copies started into each ring slot so far (the last one is waited for before the CTA leaves)
     int items[8];              // pair ids of this cluster's rounds, indexed by round & 7
     alignas(16) float tot[4];  // cluster totals of the current pair: Ka, Kb, Za, Zb
     Stats ws[kStreamWarps];    // the warps' statistics of the current pair
@@ -344,7 +350,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     const int ahead = 2 + (kRing - 2) / (ns_min > 0 ? ns_min : 1);
     if (tid == 0) {
         for (int k = 0; k < ahead; ++k) sh.items[k] = cluster_id + k * n_clusters;
-        for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kStreamWarps); }
+        for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kStreamWarps); sh.armed[s] = 0; }
         mbar_init(&sh.xbar[0], 1); mbar_init(&sh.xbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -383,6 +389,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
         const uint32_t bytes = static_cast<uint32_t>(nv) * 16;
         unsigned char* dst = ring + slot * kStageBytes;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of the slot precede the async writes
+        sh.armed[slot] += 1;                         // one thread at a time starts copies into a slot
         mbar_arrive_expect_tx(&sh.full[slot], 2 * bytes);
         bulk_g2s(dst, a_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
         bulk_g2s(dst + kStageRowBytes, b_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
@@ -523,7 +530,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
                         if (gs > 0 && warp == static_cast<int>(gs % kStreamWarps)) {
                             const uint32_t ps = gs - 1;
                             mbar_wait(&sh.empty[ps % kRing], (ps / kRing) & 1, P.timeout_flag, dead);
-                            issue_stage(ps + kRing);
+                            if (!dead) issue_stage(ps + kRing);      // after a wait has run out nothing more is copied
                         }
                     }
                     float e[VPT][EPT];
@@ -740,6 +747,19 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
 
     // ---- release tensor memory ----
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (tid == 0) {
+        // Every copy started into this CTA's ring has landed before the CTA may leave: normally the
+        // first sweep consumed them all and these waits return at once; after a wait that ran out
+        // some may still be on their way (a copy, once started, always completes).
+        for (int slot = 0; slot < kRing; ++slot) {
+            const uint32_t n = sh.armed[slot];
+            if (n == 0) continue;
+#pragma unroll 1
+            for (uint32_t i = 0; i < kSpinLimit; ++i)
+                if (mbar_try_wait(&sh.full[slot], (n - 1) & 1)) break;
+        }
+    }
     __syncthreads();
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sh.tmem_base), "r"(kTmemCols) : "memory");

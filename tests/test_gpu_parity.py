@@ -283,6 +283,20 @@ def test_chain_shaped_tree_matches_chain_call():
         assert np.array_equal(g.divergence, c.divergence)
 
 
+def test_largest_trees_chain_shaped_and_bushy():
+    """The allowed maximum of 1024 nodes: a chain-shaped tree (depth 1024, the worst case for the
+    path selection) and a bushy random one, against the oracle."""
+    N, V = 1024, 1024
+    chain_parent = np.arange(-1, N - 1, dtype=np.int32)[None, :]
+    t = gi.make_tree(2, N, V, dtype="f32", sigma=0.05, max_depth=N, workload_id=402, parent=chain_parent)
+    for T in (1e-3, 2e-3, 1.0):
+        g, o = parity.check_tree(t, T=T)
+    assert g.accept_len.max() == N                       # with T = 1 the whole chain passes
+    t = gi.make_tree(2, N, V, dtype="f32", sigma=0.3, max_depth=9, max_children=4, workload_id=403)
+    for T in (0.02, 0.05, 1.0):
+        parity.check_tree(t, T=T)
+
+
 def test_tree_max_depth_and_bad_parent():
     t = gi.make_tree(3, 12, 2048, dtype="f32", sigma=0.3, max_depth=5, workload_id=401)
     t.parent[1, 4] = 4                           # a node naming itself as parent
