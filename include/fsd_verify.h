@@ -216,6 +216,16 @@ int fsd_set_stage_event(void *event);
  * Process-wide, read when a call is made; off by default.  Returns FSD_OK. */
 int fsd_set_timeout_injection(int on);
 
+/* Debug build (no counterpart in the paper).  A library compiled with -DFSD_DEBUG_CHECKS
+ * (python -m paper_2502_20704_b200.build --debug) checks, inside its kernels, the indices and
+ * ranges behind its memory accesses -- pair ids, slice and stage bounds of the copies, tensor-
+ * memory columns, record and row indices, vocabulary chunks, token ids, tree paths -- and ORs a
+ * bit per kind of violation into one int of the workspace; the release build compiles the checks
+ * out.  Returns 1 if this library has the checks, else 0; if `word_offset` is not NULL (host
+ * pointer) and B, positions >= 1, stores the byte offset of that int inside a workspace for that
+ * shape.  The word is zero after a call in which no check failed. */
+int fsd_debug_checks(int B, int positions, size_t *word_offset);
+
 /* ---- Threshold tuning (Section "Selecting T"; Discussion, "Potential further developments") ----
  * The paper tunes T on a small development set by running FSD at candidate thresholds and
  * looking at the speed each gives, and notes that FSD's decisions are a deterministic function

@@ -5,6 +5,7 @@ from .binding import (  # noqa: F401
     FsdError,
     fsd_accept_labels,
     fsd_calibrate_threshold,
+    fsd_debug_checks,
     fsd_default_opts,
     fsd_host_staging_bytes,
     fsd_set_stage_event,

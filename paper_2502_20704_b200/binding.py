@@ -13,7 +13,8 @@ import os
 from typing import Optional
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_PKG, "lib", "libfsd_verify.so")
+# FSD_VERIFY_LIB selects another build of the same library (the debug build with range checks)
+_LIB_PATH = os.environ.get("FSD_VERIFY_LIB") or os.path.join(_PKG, "lib", "libfsd_verify.so")
 
 DIVS = {"js": 0, "kl": 1, "tv": 2}
 MODES = {"fsd": 0, "sd": 1, "rfsd": 2}
@@ -85,6 +86,8 @@ def _load():
         lib.fsd_version.restype = C.c_int
         lib.fsd_set_stage_event.argtypes = [C.c_void_p]
         lib.fsd_set_stage_event.restype = C.c_int
+        lib.fsd_debug_checks.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_size_t)]
+        lib.fsd_debug_checks.restype = C.c_int
         lib.fsd_set_timeout_injection.argtypes = [C.c_int]
         lib.fsd_set_timeout_injection.restype = C.c_int
         lib.fsd_threshold_sweep.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, C.c_int, vp, vp, C.c_void_p]
@@ -134,6 +137,13 @@ def fsd_set_stage_event(event) -> int:
     if event is not None:
         handle = getattr(event, "cuda_event", event)
     return _load().fsd_set_stage_event(handle)
+
+
+def fsd_debug_checks(B: int = 0, positions: int = 0):
+    """(enabled, byte offset of the debug word in a workspace for this shape or None)."""
+    off = C.c_size_t(0)
+    on = _load().fsd_debug_checks(int(B), int(positions), C.byref(off))
+    return bool(on), (off.value if B >= 1 and positions >= 1 else None)
 
 
 def fsd_set_timeout_injection(on: bool) -> int:

@@ -176,6 +176,9 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Pair
         fp.timeout_flag = flags;
         fp.records = records;
     } else {
+#ifdef FSD_DEBUG_CHECKS
+        if (cudaMemsetAsync(flags, 0, kAlign, s) != cudaSuccess) return FSD_ERR_CUDA;   // the debug word starts at zero here too
+#endif
         if (vec) fsd_pair_generic_kernel<DT, true><<<items, 512, 0, s>>>(pp);
         else     fsd_pair_generic_kernel<DT, false><<<items, 512, 0, s>>>(pp);
         if (cudaGetLastError() != cudaSuccess) return FSD_ERR_CUDA;
@@ -227,6 +230,7 @@ int verify_common(const void* target, const void* draft, const int32_t* tokens, 
     pp.B = B; pp.G = G; pp.V = V;
     pp.div = o->divergence; pp.mode = o->mode; pp.cmp = o->compare; pp.T = o->threshold;
     pp.divergence = divergence; pp.item_bits = ws.item_bits; pp.item_status = ws.item_status;
+    pp.debug_word = ws.flags + 2;
 
     FinishParams fp;
     fp.target = target; fp.draft = draft; fp.parent = parent; fp.u_sample = u_sample;
@@ -236,6 +240,7 @@ int verify_common(const void* target, const void* draft, const int32_t* tokens, 
     fp.T = o->threshold; fp.records = nullptr; fp.divergence = divergence;
     fp.item_bits = ws.item_bits; fp.item_status = ws.item_status; fp.timeout_flag = nullptr;
     fp.accept_len = accept_len; fp.path = path; fp.next_token = next_token; fp.row_status = row_status;
+    fp.debug_word = ws.flags + 2;
 
     const bool vec = (static_cast<size_t>(V) * es) % 16 == 0 && aligned(target, 16) && aligned(draft, 16);
     fp.vec = vec ? 1 : 0;
@@ -440,6 +445,18 @@ int fsd_version(void) { return 100; }
 int fsd_set_stage_event(void* event) {
     g_stage_event.store(event);
     return FSD_OK;
+}
+
+int fsd_debug_checks(int B, int positions, size_t* word_offset) {
+    if (word_offset != nullptr && B >= 1 && positions >= 1) {
+        const Workspace w = carve(nullptr, B, positions);
+        *word_offset = static_cast<size_t>(reinterpret_cast<char*>(w.flags + 2) - static_cast<char*>(nullptr));
+    }
+#ifdef FSD_DEBUG_CHECKS
+    return 1;
+#else
+    return 0;
+#endif
 }
 
 int fsd_set_timeout_injection(int on) {

@@ -8,9 +8,23 @@
 
 #include "fsd_verify.h"
 
+// Index and range checks of the debug build (-DFSD_DEBUG_CHECKS, see build.py): a failed check
+// sets a bit in the workspace's debug word and the access goes ahead as in the release build --
+// the checks are there to show that it never happens, on inputs of every shape the tests run.
+// `word` is the third int of the workspace's flag block; null disables the check.
+#ifdef FSD_DEBUG_CHECKS
+#define FSD_CHECK(word, cond, code) do { if ((word) != nullptr && !(cond)) atomicOr((word), (code)); } while (0)
+#else
+#define FSD_CHECK(word, cond, code) do { } while (0)
+#endif
+
 namespace fsd {
 
 namespace cg = cooperative_groups;
+
+// bits of the debug word
+constexpr int kChkItem = 1, kChkSlice = 2, kChkStage = 4, kChkTmem = 8, kChkRecord = 16, kChkRow = 32, kChkChunk = 64,
+              kChkToken = 128, kChkPath = 256;
 
 constexpr float  kLog2e  = 1.4426950408889634f;
 constexpr double kLog2eD = 1.4426950408889634074;

@@ -47,6 +47,7 @@ struct FinishParams {
     int32_t* path;             // [B, max_depth] (tree) or null
     int32_t* next_token;       // [B]
     int32_t* row_status;       // [B]
+    int* debug_word;           // debug build: where failed range checks are recorded (may be null)
 };
 
 struct FinishExchange {        // what one CTA publishes to its cluster
@@ -372,9 +373,12 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     } else {
         tree_select(P.parent + static_cast<size_t>(b) * G, G, P.max_depth,
                     rank == 0 ? P.path + static_cast<size_t>(b) * P.max_depth : nullptr, sh);
+        __syncthreads();
+        FSD_CHECK(P.debug_word, sh.row_sel >= 0 && sh.row_sel <= G && sh.n_acc >= 0 && sh.n_acc <= P.max_depth, kChkPath);
     }
     __syncthreads();
     const int n = sh.n_acc, row_sel = sh.row_sel;
+    FSD_CHECK(P.debug_word, row_sel >= 0 && row_sel <= G && n >= 0 && n <= (tree ? P.max_depth : G), kChkRow);
     int status = sh.bad;
     if (status & FSD_ROW_BADTREE) {                      // uniform over the cluster
         if (rank == 0 && tid == 0) { P.accept_len[b] = 0; P.next_token[b] = -1; P.row_status[b] = status; }
@@ -396,6 +400,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const long long k0l = static_cast<long long>(rank * blockDim.x + tid) * L;
     const int k0 = k0l < V ? static_cast<int>(k0l) : V;
     const int k1 = (k0l + L) < V ? static_cast<int>(k0l + L) : V;
+    FSD_CHECK(P.debug_word, k0 >= 0 && k0 <= k1 && k1 <= V && (!vec || k0 % EPV == 0), kChkChunk);
     FinishExchange mine;
     FinishExchange* const all = sh.all;
     double* const sc = sh.sc;
@@ -530,6 +535,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             }
             tok = __reduce_min_sync(0xffffffffu, tok);
             lastp = __reduce_max_sync(0xffffffffu, lastp);
+            FSD_CHECK(P.debug_word, (tok != 0x7fffffff ? tok : lastp) >= -1 && (tok != 0x7fffffff ? tok : lastp) < V, kChkToken);
             if (lane == 0) P.next_token[b] = tok != 0x7fffffff ? tok : lastp;
         }
         return;
@@ -776,6 +782,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                 base = __shfl_sync(0xffffffffu, run, 31);
             }
             tok = __reduce_min_sync(0xffffffffu, tok);
+            FSD_CHECK(P.debug_word, (tok != 0x7fffffff ? tok : fallback) >= -1 && (tok != 0x7fffffff ? tok : fallback) < V, kChkToken);
             if (lane == 0) P.next_token[b] = tok != 0x7fffffff ? tok : fallback;
         }
         return;

@@ -22,6 +22,7 @@ struct PairParams {
     float* divergence;         // [B, G]
     int32_t* item_bits;        // [B, G] accept bit per pair
     int32_t* item_status;      // [B, G] FSD_ROW_* flags per pair
+    int* debug_word;           // debug build: where failed range checks are recorded (may be null)
 };
 
 // Final scalar work for one pair, done by one thread in double precision.
@@ -188,6 +189,7 @@ __global__ void __launch_bounds__(512) fsd_pair_generic_kernel(PairParams P) {
 
     const int item = blockIdx.x;
     const int b = item / P.G, i = item - b * P.G;
+    FSD_CHECK(P.debug_word, b < P.B, kChkItem);
     int trow = i;
     if (P.parent != nullptr) {
         const int par = P.parent[item];

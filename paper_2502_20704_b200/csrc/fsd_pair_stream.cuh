@@ -375,6 +375,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
         const uint32_t k = gg / static_cast<uint32_t>(ns), s = gg - k * static_cast<uint32_t>(ns);
         const int item = sh.items[k & 7];
         if (item >= P.n_items) return;
+        FSD_CHECK(P.timeout_flag + 2, item >= 0, kChkItem);
         const int b = item / P.G, i = item - b * P.G;
         int trow = i;
         if (P.parent != nullptr) {
@@ -387,6 +388,8 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
         const int v0 = static_cast<int>(s) * kStageVecs;
         const int nv = (vcnt - v0) < kStageVecs ? (vcnt - v0) : kStageVecs;
         const uint32_t bytes = static_cast<uint32_t>(nv) * 16;
+        FSD_CHECK(P.timeout_flag + 2, nv > 0 && vbeg + v0 + nv <= P.nvec_row && bytes <= kStageRowBytes, kChkSlice);
+        FSD_CHECK(P.timeout_flag + 2, s < static_cast<uint32_t>(ns) && ns <= kMaxStagesPerPair && trow >= 0 && trow <= P.G, kChkStage);
         unsigned char* dst = ring + slot * kStageBytes;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of the slot precede the async writes
         sh.armed[slot] += 1;                         // one thread at a time starts copies into a slot
@@ -575,6 +578,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
 #pragma unroll
                         for (int v = 0; v < VPT; ++v) {
                             if (s < NT) {
+                                FSD_CHECK(P.timeout_flag + 2, (s * VPT + v) * EPT + EPT <= kTmemPerThread, kChkTmem);
                                 tmem_st<EPT>(taddr + (s * VPT + v) * EPT, e[v]);
                             } else {
 #pragma unroll
@@ -673,6 +677,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
             if (rank == 0 && lane < C) {
                 if (prev_item >= 0) P.records[prev_item].x[lane] = t.x;
                 if (live) {
+                    FSD_CHECK(P.timeout_flag + 2, item >= 0 && item < P.n_items && C <= kStreamMaxCluster, kChkRecord);
                     PairRecord* r = P.records + item;
                     r->part[lane] = t;
                     if (lane == 0) { r->ncta = static_cast<uint32_t>(C); r->state = bad ? kRecordBadTree : kRecordStats; }

@@ -116,3 +116,10 @@ def test_tuning_entry_points_check_their_arguments_on_the_host():
     assert fsd.fsd_calibrate_threshold(None, 1, 1, 1.0, 0, 16, 16) == -1
     assert fsd.fsd_accept_labels(16, 1, 0, 0.1, 1, 16) == -2
     assert fsd.fsd_accept_labels(16, 1, 1, 0.1, 2, 16) == -4
+
+
+def test_release_build_reports_no_debug_checks_and_a_word_inside_the_workspace():
+    import paper_2502_20704_b200 as fsd
+    on, off = fsd.fsd_debug_checks(4, 8)
+    assert on is False
+    assert 0 < off < fsd.fsd_workspace_bytes(4, 8, 32000, fsd.make_opts(T=0.1))
