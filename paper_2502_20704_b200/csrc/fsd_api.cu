@@ -18,6 +18,8 @@ namespace {
 using namespace fsd;
 
 constexpr size_t kAlign = 256;
+constexpr int kMaxVirtualCtas = 512;                                   // two per SM
+constexpr size_t kExchangeBytes = 2 * kMaxVirtualCtas * sizeof(GroupMsg);
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -25,6 +27,7 @@ struct Workspace {
     int32_t* item_bits;
     int32_t* item_status;
     int* flags;                // [0] = a bounded device-side wait ran out
+    GroupMsg* exchange;        // the streaming kernel's statistics exchange (directly after the flags: one memset clears both)
     PairRecord* records;       // per-pair totals of the streaming kernel
     size_t bytes;
 };
@@ -39,6 +42,8 @@ Workspace carve(void* base, int B, int G) {
     p += align_up(items * sizeof(int32_t));
     w.flags = reinterpret_cast<int*>(p);
     p += kAlign;
+    w.exchange = reinterpret_cast<GroupMsg*>(p);
+    p += kExchangeBytes;
     w.records = reinterpret_cast<PairRecord*>(p);
     p += align_up(items * sizeof(PairRecord));
     w.bytes = static_cast<size_t>(p - static_cast<char*>(base));
@@ -79,97 +84,97 @@ std::atomic<int> g_mark_timeout{0};          // see fsd_set_timeout_injection
 // ---- streaming kernel launch -----------------------------------------------------------
 constexpr int kMaxDev = 64;
 
-inline void stream_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int C, cudaStream_t s) {
-    cfg = {};
-    cfg.blockDim = dim3(kStreamThreads, 1, 1);
-    cfg.dynamicSmemBytes = kStreamSmemBytes;
-    cfg.stream = s;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = C;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-}
-
-// Attributes of the kernel and the number of clusters that can be resident (cached per device and
-// cluster size).  Puts nothing on a stream.
+// One CTA of two virtual CTAs per SM, all resident (cooperative launch).  Puts nothing on a stream.
 template <int DT, int DIV>
-int prepare_stream(int C, int* nclus_out) {
-    static int max_clusters[kMaxDev][5] = {};       // per device, per log2(C); 0 = not yet queried
+int prepare_stream(int dev) {
+    static bool ready[kMaxDev] = {};
     static std::mutex mu;
     auto kernel = fsd_pair_stream_kernel<DT, DIV>;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return FSD_ERR_CUDA;
-    int lc = 0;
-    while ((1 << lc) < C) ++lc;
+    if (dev < 0 || dev >= kMaxDev) return FSD_ERR_CUDA;
     std::lock_guard<std::mutex> lock(mu);
-    if (max_clusters[dev][lc] == 0) {
+    if (!ready[dev]) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
             return FSD_ERR_CUDA;
-        if (cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kStreamSmemBytes)) != cudaSuccess)
+        int per = 0;                                 // one CTA must fit an SM, or the cooperative launch is refused
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, kernel, kStreamCtaThreads, kStreamSmemBytes) != cudaSuccess || per < 1)
             return FSD_ERR_CUDA;
-        if (C > 8) {                            // above the portable cluster size: opt in
-            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-                cudaFuncSetAttribute(fsd_stream_occupancy_twin, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
-                return FSD_ERR_CUDA;
-        }
-        cudaLaunchConfig_t cfg;
-        cudaLaunchAttribute attr[1];
-        stream_config(cfg, attr, C, nullptr);
-        cfg.gridDim = dim3(C, 1, 1);
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, fsd_stream_occupancy_twin, &cfg) != cudaSuccess || n < 1)
-            return FSD_ERR_CUDA;
-        max_clusters[dev][lc] = n;
+        ready[dev] = true;
     }
-    *nclus_out = max_clusters[dev][lc];
     return FSD_OK;
 }
 
 template <int DT, int DIV>
-int launch_stream(const StreamParams& sp, int C, int nclus, cudaStream_t s) {
-    cudaLaunchConfig_t cfg;
+int launch_stream(const StreamParams& gp, int nsm, cudaStream_t s) {
+    // as many CTAs as give every pair a group, at most one per SM and what the exchange buffer holds
+    long long want = (static_cast<long long>(gp.n_items) * gp.C + kStreamHalves - 1) / kStreamHalves;
+    int grid = nsm;
+    if (grid > kMaxVirtualCtas / kStreamHalves) grid = kMaxVirtualCtas / kStreamHalves;
+    if (want < grid) grid = static_cast<int>(want);
+    if (grid * kStreamHalves < gp.C) return FSD_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kStreamCtaThreads, 1, 1);
+    cfg.dynamicSmemBytes = kStreamSmemBytes;
+    cfg.stream = s;
     cudaLaunchAttribute attr[1];
-    stream_config(cfg, attr, C, s);
-    if (nclus > sp.n_items) nclus = sp.n_items;
-    cfg.gridDim = dim3(static_cast<unsigned>(nclus) * C, 1, 1);
-    if (cudaLaunchKernelEx(&cfg, fsd_pair_stream_kernel<DT, DIV>, sp) != cudaSuccess) return FSD_ERR_CUDA;
+    attr[0].id = cudaLaunchAttributeCooperative;     // the groups' virtual CTAs wait for one another: all must be resident
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, fsd_pair_stream_kernel<DT, DIV>, gp) != cudaSuccess) return FSD_ERR_CUDA;
     return FSD_OK;
 }
 
-// Cluster size for the streaming kernel: the smallest power of two whose per-CTA slice fits
-// on chip; 0 if the shape is not eligible (the generic kernel takes it).
-int stream_cluster_size(int nvec_row, bool vec) {
+// Virtual CTAs per pair for the streaming kernel; 0 if the shape is not eligible (the generic
+// kernel takes it).  Between the fewest whose slice fits on chip and kMaxGroupSize it is the size
+// with the lowest estimated time -- rounds * (fixed cost of a round +
+// cost of a ring stage * stages per slice), the two costs (3.4 and 1.07 us) measured on a B200.
+// Few pairs are spread over many virtual CTAs (short rounds); many pairs over few (fewer rounds).
+int group_size(int nvec_row, bool vec, int items, int nsm) {
     if (!vec || nvec_row < 64) return 0;
-    for (int C = 1; C <= kStreamMaxCluster; C <<= 1)
-        if ((nvec_row + C - 1) / C <= kMaxVecPerCta) return C;
-    return 0;
+    const int cmin = (nvec_row + kMaxVecPerCta - 1) / kMaxVecPerCta;
+    int vctas = kStreamHalves * nsm;
+    if (vctas > kMaxVirtualCtas) vctas = kMaxVirtualCtas;
+    int best = 0;
+    double best_cost = 0.0;
+    for (int C = cmin; C <= kMaxGroupSize && C <= vctas; ++C) {
+        const int groups = vctas / C;
+        const int rounds = (items + groups - 1) / groups;
+        const int slice = (nvec_row + C - 1) / C;
+        const int stages = (slice + kStageVecs - 1) / kStageVecs;
+        const double cost = rounds * (3.4 + 1.07 * stages);
+        if (best == 0 || cost < best_cost) { best = C; best_cost = cost; }
+    }
+    return best;
 }
 
 template <int DT>
-int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, PairRecord* records, cudaStream_t s) {
+int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, GroupMsg* exchange, PairRecord* records, cudaStream_t s) {
     const int items = pp.B * pp.G;
     const int nvec_row = pp.V / Logit<DT>::kPerVec;
-    const int C = stream_cluster_size(nvec_row, vec);
+    int dev = 0, nsm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || nsm < 1)
+        return FSD_ERR_CUDA;
+    const int C = group_size(nvec_row, vec, items, nsm);
     if (C > 0) {
         StreamParams sp;
         sp.target = pp.target; sp.draft = pp.draft; sp.parent = pp.parent; sp.B = pp.B; sp.G = pp.G;
         sp.nvec_row = nvec_row; sp.n_items = items; sp.records = records; sp.timeout_flag = flags; sp.next_pair = flags + 1;
+        sp.C = C; sp.exchange = exchange;
         // everything that can fail without a launch (attributes, the occupancy query) comes before
         // the first thing put on the stream
-        int rc, nclus = 0;
-        if (pp.div == FSD_DIV_JS)      rc = prepare_stream<DT, FSD_DIV_JS>(C, &nclus);
-        else if (pp.div == FSD_DIV_KL) rc = prepare_stream<DT, FSD_DIV_KL>(C, &nclus);
-        else                           rc = prepare_stream<DT, FSD_DIV_TV>(C, &nclus);
+        int rc;
+        if (pp.div == FSD_DIV_JS)      rc = prepare_stream<DT, FSD_DIV_JS>(dev);
+        else if (pp.div == FSD_DIV_KL) rc = prepare_stream<DT, FSD_DIV_KL>(dev);
+        else                           rc = prepare_stream<DT, FSD_DIV_TV>(dev);
         if (rc != FSD_OK) return rc;
-        // the flag block starts every call at zero: [0] timeout, [1] pairs handed out
-        if (cudaMemsetAsync(flags, 0, kAlign, s) != cudaSuccess) return FSD_ERR_CUDA;
-        if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, C, nclus, s);
-        else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, C, nclus, s);
-        else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, C, nclus, s);
+        // the flag block and the exchange buffer start every call at zero: flags [0] timeout, [1] pairs handed out
+        if (cudaMemsetAsync(flags, 0, kAlign + kExchangeBytes, s) != cudaSuccess) return FSD_ERR_CUDA;
+        if (pp.div == FSD_DIV_JS)      rc = launch_stream<DT, FSD_DIV_JS>(sp, nsm, s);
+        else if (pp.div == FSD_DIV_KL) rc = launch_stream<DT, FSD_DIV_KL>(sp, nsm, s);
+        else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, nsm, s);
         if (rc != FSD_OK) return rc;
         // test aid: behave as if a bounded wait of the streaming kernel had run out
         if (g_mark_timeout.load() != 0 && cudaMemsetAsync(flags, 1, sizeof(int), s) != cudaSuccess) return FSD_ERR_CUDA;
@@ -245,8 +250,8 @@ int verify_common(const void* target, const void* draft, const int32_t* tokens, 
     const bool vec = (static_cast<size_t>(V) * es) % 16 == 0 && aligned(target, 16) && aligned(draft, 16);
     fp.vec = vec ? 1 : 0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, ws.flags, ws.records, s)
-                                       : launch_all<FSD_F32>(pp, fp, vec, ws.flags, ws.records, s);
+    return o->logit_dtype == FSD_BF16 ? launch_all<FSD_BF16>(pp, fp, vec, ws.flags, ws.exchange, ws.records, s)
+                                       : launch_all<FSD_F32>(pp, fp, vec, ws.flags, ws.exchange, ws.records, s);
 }
 
 struct HostStaging {

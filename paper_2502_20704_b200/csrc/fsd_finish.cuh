@@ -122,7 +122,7 @@ __device__ __forceinline__ void cluster_gather(cg::cluster_group& cluster, Finis
 }
 
 // Divergence, accept bit and status of one pair from the streaming kernel's totals.
-// A pair's totals from the parts its record holds (one per CTA of the streaming cluster), in
+// A pair's totals from the parts its record holds (one per virtual CTA of the streaming group), in
 // double: Z = sum 2^y, S = sum 2^y * y, K = sum 2^ya (ya - yb), all relative to the largest
 // part reference (the parts' references are integers, so the factors are exact powers of two).
 struct PairTotals {
@@ -134,15 +134,15 @@ struct PairTotals {
 __device__ __forceinline__ double pow2_int_d(double d) {
     return d < -1022.0 ? 0.0 : __hiloint2double((1023 + static_cast<int>(d)) << 20, 0);
 }
-__device__ __forceinline__ double group_sum(double v) {       // over the kStreamMaxCluster lanes of a record
+__device__ __forceinline__ double group_sum(double v) {       // over the kMaxGroupSize lanes of a record
 #pragma unroll
-    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+    for (int m = kMaxGroupSize / 2; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
     return v;
 }
 // Called by all 32 lanes: lane 16*q + r folds part r of the record `rec` of group q (null: no
 // record for this group); every lane of a group returns the group's totals.
 __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
-    const int r = threadIdx.x & (kStreamMaxCluster - 1);
+    const int r = threadIdx.x & (kMaxGroupSize - 1);
     PairTotals t;
     Stats c;
     c.ka = -INFINITY; c.kb = -INFINITY; c.za = 0.f; c.zb = 0.f; c.s0 = 0.f; c.sb = 0.f; c.x = 0.f; c.diff = 0;
@@ -150,7 +150,7 @@ __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     if (rec != nullptr && r < static_cast<int>(rec->ncta)) { c = rec->part[r]; x = rec->x[r]; }
     float ka = c.ka, kb = c.kb;                          // NaN references win
 #pragma unroll
-    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) {
+    for (int m = kMaxGroupSize / 2; m > 0; m >>= 1) {
         const float oa = __shfl_xor_sync(0xffffffffu, ka, m), ob = __shfl_xor_sync(0xffffffffu, kb, m);
         ka = (oa != oa || ka != ka) ? __int_as_float(0x7fc00000) : fmaxf(ka, oa);
         kb = (ob != ob || kb != kb) ? __int_as_float(0x7fc00000) : fmaxf(kb, ob);
@@ -175,7 +175,7 @@ __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     t.X = group_sum(static_cast<double>(x));
     uint32_t df = c.diff;
 #pragma unroll
-    for (int m = kStreamMaxCluster / 2; m > 0; m >>= 1) df |= __shfl_xor_sync(0xffffffffu, df, m);
+    for (int m = kMaxGroupSize / 2; m > 0; m >>= 1) df |= __shfl_xor_sync(0xffffffffu, df, m);
     t.differ = df;
     return t;
 }
@@ -419,14 +419,14 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             if (r->state & kRecordStats) {
                 float rka = -INFINITY;
                 bool nan = false;
-                for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
+                for (uint32_t c = 0; c < r->ncta && c < kMaxGroupSize; ++c) {
                     const float a = r->part[c].ka;
                     nan = nan || a != a;
                     rka = fmaxf(rka, a);
                 }
                 if (!nan && isfinite(rka)) {
                     float za = 0.f;
-                    for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
+                    for (uint32_t c = 0; c < r->ncta && c < kMaxGroupSize; ++c) {
                         const float a = r->part[c].ka;
                         if (a != -INFINITY) za += r->part[c].za * pow2_int(a - rka);
                     }
@@ -552,7 +552,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         if (r->state & kRecordStats) {
             float fa = -INFINITY, fb = -INFINITY;
             bool nan = false;
-            for (uint32_t c = 0; c < r->ncta && c < kStreamMaxCluster; ++c) {
+            for (uint32_t c = 0; c < r->ncta && c < kMaxGroupSize; ++c) {
                 const float a = r->part[c].ka, q = r->part[c].kb;
                 nan = nan || a != a || q != q;
                 fa = fmaxf(fa, a); fb = fmaxf(fb, q);

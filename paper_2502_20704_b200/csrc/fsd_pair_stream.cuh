@@ -1,8 +1,12 @@
 // Streaming per-(row, position) kernel: every logit is read from HBM once.
 //
-// A (row, position) pair is split along the vocabulary over a thread-block cluster of C CTAs
-// (C = 1, 2, 4, 8 or 16, the smallest that lets a CTA's slice fit on chip).  Clusters are
-// persistent and claim pairs from a shared counter.  Per pair, each CTA
+// A (row, position) pair is split along the vocabulary over a GROUP of C virtual CTAs (C <= 16,
+// chosen by the host from the slice that fits on chip and the number of pairs).  A CTA of 512
+// threads, one per SM, holds two virtual CTAs of 256 threads, each with its own half of the SM's
+// tensor memory, its own shared-memory ring and its own named barriers; the two belong to
+// different groups, so that one computes while the other waits for its group.  The launch is
+// cooperative (all CTAs resident: the virtual CTAs of a group wait for one another) and the groups
+// are persistent: they claim pairs from a shared counter.  Per pair, each virtual CTA
 //   1. receives its slice of both rows in shared memory through a ring of bulk asynchronous
 //      copies (cp.async.bulk + mbarrier).  A warp releases a slot as soon as its vectors are in
 //      registers; the slot is refilled one stage later by a rotating duty warp, so the next
@@ -14,19 +18,20 @@
 //      logits and moved -- with an exact power-of-two rescale of what has been summed and parked
 //      -- only if a later logit exceeds it by more than 2^30, so no separate maximum pass over
 //      the slice is needed and every change of reference is exact;
-//   3. combines (k, Z, S) over threads and warps; one combiner warp per CTA (rotating) folds
-//      the warps' statistics, sends them to every CTA of the cluster with asynchronous
-//      distributed-shared-memory stores that signal the receiver's mbarrier, folds what the
-//      cluster sent and wakes the CTA (named barriers: waiting warps issue nothing);
+//   3. combines (k, Z, S) over threads and warps; one combiner warp per virtual CTA (rotating)
+//      folds the warps' statistics, leaves them as a tagged message in global memory, fetches the
+//      messages of the whole group (they live in L2), folds those and wakes the virtual CTA
+//      (named barriers: waiting warps issue nothing);
 //   4. sweeps the parked e values: p = e_a/Z_a, q = e_b/Z_b; JS needs sum (p+q) log2(p+q) (one
 //      MUFU lg2 per pair), TV needs sum |p - q|; KL needs no second sweep.
-// The cluster's rank-0 CTA leaves the CTAs' statistics in the pair's record; the finish kernel
-// folds them in double precision and turns them into divergences and accept bits, so no
+// The group's rank-0 virtual CTA leaves all members' statistics in the pair's record; the finish
+// kernel folds them in double precision and turns them into divergences and accept bits, so no
 // double-precision arithmetic runs here.  HBM traffic is the algorithmic minimum.  The
 // special-function pipe (1 ex2 per logit + 1 lg2 per pair) and instruction issue are the
 // co-bottlenecks, which is why e values are kept rather than recomputed, and why a thread
-// owns two vectors per row and stage (independent work to overlap its own latencies) with two
-// CTAs of 256 threads and 128 registers per SM.
+// owns two vectors per row and stage (independent work to overlap its own latencies) with 512
+// threads of 128 registers per SM.  Groups need no co-scheduling on neighbouring SMs, so every
+// SM is used whatever C is.
 #pragma once
 
 #include "fsd_device.cuh"
@@ -41,16 +46,15 @@ constexpr int kStageVecs = kStreamThreads * kVecPerThread; // vectors per row an
 constexpr int kStageRowBytes = kStageVecs * 16;
 constexpr int kStageBytes = 2 * kStageRowBytes;
 constexpr int kMaxStagesPerPair = kRing - 1;               // stages of e values a thread can park (4 in tensor memory, 1 in registers)
-constexpr int kTmemCols = 256;                             // per CTA: 8 warps -> 2 per lane quarter x 128 columns
+constexpr int kTmemCols = 256;                             // per virtual CTA: 8 warps -> 2 per lane quarter x 128 columns
 constexpr int kTmemPerThread = 128;
 constexpr int kMaxVecPerCta = kMaxStagesPerPair * kStageVecs;
 constexpr int kMaxClusterSize = 8;                        // finish kernel (portable size)
-constexpr int kStreamMaxCluster = 16;                      // streaming kernel (above 8: the non-portable opt-in)
-constexpr int kStreamCtasPerSm = 2;
+constexpr int kMaxGroupSize = 16;                      // most virtual CTAs in a group of the streaming kernel
 constexpr uint32_t kSpinLimit = 1u << 24;                  // polls before a wait gives up
 
-// Partial statistics of one (target row, draft row) pair: of a warp, of a CTA, or -- in a
-// pair's record -- of each CTA of the cluster that streamed the pair.
+// Partial statistics of one (target row, draft row) pair: of a warp, of a virtual CTA, or -- in a
+// pair's record -- of each virtual CTA of the group that streamed the pair.
 //   z = sum 2^y, s = sum 2^y * y with y = logit*log2e - k and k the integer reference (log2
 //   domain) the sums are relative to.  s0 is the target row's s for JS and the KL sum
 //   sum 2^ya (ya - yb) for KL.
@@ -59,22 +63,31 @@ struct alignas(16) Stats {
     float za, zb;
     float s0, sb;
     float x;                   // second-sweep sum of the PREVIOUS pair (in flight only)
-    uint32_t diff;             // 0: the two rows are bitwise identical so far (bit 0 once a CTA has folded it;
-                               // rank 0's message carries the next claimed pair id in the bits above)
+    uint32_t diff;             // 0: the two rows are bitwise identical so far (bit 0 once a virtual CTA has folded
+                               // it; rank 0's message carries the next claimed pair id in the bits above)
 };
 static_assert(sizeof(Stats) == 32, "Stats travels as two 16-byte stores");
 
 // What the streaming kernel leaves per pair for the finish kernel, which folds the parts in
 // double precision (second-sweep sums: JS sum s log2 s, TV sum |p - q|).
 struct alignas(16) PairRecord {
-    Stats part[kStreamMaxCluster];
-    float x[kStreamMaxCluster];  // each CTA's second-sweep sum of this pair
+    Stats part[kMaxGroupSize];
+    float x[kMaxGroupSize];  // each virtual CTA's second-sweep sum of this pair
     uint32_t ncta;             // parts in use
     uint32_t state;            // kRecordStats | kRecordBadTree
     uint32_t pad[2];
 };
 static_assert(sizeof(PairRecord) == 592, "PairRecord layout");
 constexpr uint32_t kRecordStats = 1, kRecordBadTree = 2;
+
+// One virtual CTA's statistics of a round as they cross global memory: three 16-byte units, each
+// stored whole and ending in the round's tag, so that a reader knows a unit is this round's
+// without any fence or flag (a unit whose tag is older is fetched again).
+struct alignas(16) GroupMsg {
+    uint4 u[3];                // {ka, kb, za, tag}, {zb, s0, sb, tag}, {x, diff | next pair id << 1, 0, tag}
+    uint4 pad;
+};
+static_assert(sizeof(GroupMsg) == 64, "GroupMsg layout");
 
 struct StreamParams {
     const void* target;        // [B, G+1, V]
@@ -85,7 +98,9 @@ struct StreamParams {
     int n_items;               // B * G
     PairRecord* records;       // [B * G]
     int* timeout_flag;         // set to 1 if a bounded wait ran out; zero at launch
-    int* next_pair;            // pairs handed out beyond each cluster's fixed first ones; zero at launch
+    int* next_pair;            // pairs handed out beyond each group's fixed first ones; zero at launch
+    int C;                     // virtual CTAs per group (<= kMaxGroupSize)
+    GroupMsg* exchange;        // [groups][2][C], zero at launch
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -253,18 +268,9 @@ __device__ __noinline__ void rescale_parked(uint32_t taddr, int n, float fa, flo
 // when the factor underflows to 0
 __device__ __forceinline__ float scale_kl(float f, float v) { return v == INFINITY ? v : f * v; }
 
-// 16-byte store into CTA `rank`'s copy of `dst` that, on landing, counts 16 bytes on that CTA's
-// copy of barrier `bar`: the store carries its own signal, the sender neither fences nor waits
-__device__ __forceinline__ void st_async_remote(void* dst, uint64_t* bar, uint32_t rank, float a, float b, float c, float d) {
-    uint32_t rdst, rbar;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rdst) : "r"(smem_u32(dst)), "r"(rank));
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(bar)), "r"(rank));
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
-                 ::"r"(rdst), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)), "r"(__float_as_uint(d)), "r"(rbar)
-                 : "memory");
-}
-// CTA-wide named barriers: waiting warps issue nothing.  `arrive` counts the warp in without
-// waiting; `sync` waits until kStreamThreads threads have arrived or synced.
+// Named barriers of one virtual CTA: waiting warps issue nothing.  `arrive` counts the warp in
+// without waiting; `sync` waits until kStreamThreads threads have arrived or synced.  The second
+// virtual CTA of a CTA uses ids two higher.
 __device__ __forceinline__ void named_arrive(int id) {
     asm volatile("bar.arrive %0, %1;" ::"r"(id), "n"(kStreamThreads) : "memory");
 }
@@ -273,44 +279,32 @@ __device__ __forceinline__ void named_sync(int id) {
 }
 constexpr int kBarPosted = 1, kBarTotals = 2;
 
-// ---- cluster-scope mbarrier wait (the statistics exchange) ------------------------------------
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
+__device__ __forceinline__ void st_unit(uint4* p, float a, float b, float c, uint32_t tag) {
+    asm volatile("st.relaxed.gpu.global.v4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"l"(p), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)), "r"(tag) : "memory");
 }
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, int* timeout_flag, bool& dead) {
-    if (dead) return false;
-#pragma unroll 1
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int*>(timeout_flag) != 0) break;
-    }
-    atomicExch(timeout_flag, 1);
-    dead = true;
-    return false;
+__device__ __forceinline__ uint4 ld_unit(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.relaxed.gpu.global.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
 }
 
 // ---- shared-memory layout ---------------------------------------------------------------
 struct StreamShared {
     uint64_t full[kRing];      // a ring stage has landed
-    uint64_t xbar[2];          // all CTAs' statistics have landed here (per parity): 1 arrival + C * 32 bytes
     uint64_t empty[kRing];     // every warp has finished reading the slot's current stage
-    uint32_t tmem_base;
-    uint32_t armed[kRing];     // copies started into each ring slot so far (the last one is waited for before the CTA leaves)
-    int items[8];              // pair ids of this cluster's rounds, indexed by round & 7
-    alignas(16) float tot[4];  // cluster totals of the current pair: Ka, Kb, Za, Zb
+    uint32_t armed[kRing];     // copies started into each ring slot so far (the last one is waited for before leaving)
+    int items[8];              // pair ids of this group's rounds, indexed by round & 7
+    alignas(16) float tot[4];  // group totals of the current pair: Ka, Kb, Za, Zb
     Stats ws[kStreamWarps];    // the warps' statistics of the current pair
-    Stats xch[2][kStreamMaxCluster];         // written by the peers (and by this CTA for its own rank)
 };
-constexpr size_t kStreamSmemBytes = kRing * kStageBytes + sizeof(StreamShared) + 128;
+constexpr int kStreamHalves = 2;                            // virtual CTAs per CTA
+constexpr int kStreamCtaThreads = kStreamHalves * kStreamThreads;
+constexpr size_t kStreamHalfBytes = kRing * kStageBytes + ((sizeof(StreamShared) + 127) / 128) * 128;
+constexpr size_t kStreamSmemBytes = kStreamHalves * kStreamHalfBytes + 128 + 16;
 
 template <int DT, int DIV>
-__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_stream_kernel(StreamParams P) {
+__global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(StreamParams P) {
     constexpr int EPV = Logit<DT>::kPerVec;          // logits per 16-byte vector
     constexpr int EPT = 2 * EPV;                     // e values per thread and vector position (both rows)
     constexpr int VPT = kVecPerThread;
@@ -321,16 +315,23 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     constexpr float kClamp = -1.0e30f;               // -inf logits are read as this: 2^y = 0 and 0 * y = 0 stay finite
 
     extern __shared__ unsigned char smem_raw[];
-    unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    const int half = threadIdx.x / kStreamThreads;   // which virtual CTA of this CTA
+    unsigned char* ring = smem + half * kStreamHalfBytes;
     StreamShared& sh = *reinterpret_cast<StreamShared*>(ring + kRing * kStageBytes);
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + kStreamHalves * kStreamHalfBytes);
 
-    cg::cluster_group cluster = cg::this_cluster();
-    const int C = static_cast<int>(cluster.num_blocks());
-    const int rank = static_cast<int>(cluster.block_rank());
-    const int cluster_id = blockIdx.x / C, n_clusters = gridDim.x / C;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int C = P.C;
+    // numbered half by half, so that the two virtual CTAs of an SM belong to different groups: while one
+    // waits for its group's statistics the other has the SM to itself
+    const int vid = half * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int n_groups = (kStreamHalves * static_cast<int>(gridDim.x)) / C;     // groups
+    const int group_id = vid / C, rank = vid - group_id * C;
+    const bool active = group_id < n_groups;     // the virtual CTAs left over form no group
+    const int tid = threadIdx.x % kStreamThreads, lane = tid & 31, warp = tid >> 5;
+    const int bar_posted = kBarPosted + 2 * half, bar_totals = kBarTotals + 2 * half;
 
-    // this CTA's slice of every row, in vectors
+    // this virtual CTA's slice of every row, in vectors
     const int base = P.nvec_row / C, rem = P.nvec_row % C;
     const int vbeg = rank * base + (rank < rem ? rank : rem);
     const int vcnt = base + (rank < rem ? 1 : 0);
@@ -338,37 +339,39 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     const size_t row_bytes = static_cast<size_t>(P.nvec_row) * 16;
 
     // ---- set-up: barriers, tensor memory ----
-    // A cluster's first `ahead` pairs are fixed (cluster_id + round * n_clusters): that is as far
+    // A group's first `ahead` pairs are fixed (group_id + round * n_groups): that is as far
     // as the ring reads ahead.  Every later pair is the next one nobody has taken yet, claimed
-    // `ahead` rounds early by rank 0 and sent round with that round's statistics, so clusters
+    // `ahead` rounds early by rank 0 and sent round with that round's statistics, so groups
     // that happen to run faster take more pairs and all finish together.
-    // (from the smallest slice of the cluster, so that every CTA of the cluster computes the same
-    // value whatever its own slice: the CTAs must agree on which pairs are fixed and where a claimed
-    // id is kept; a CTA with one stage more per pair reads ahead less far, so the ids it needs are
-    // there even earlier)
+    // (from the smallest slice of the group, so that every member computes the same value
+    // whatever its own slice: the members must agree on which pairs are fixed and where a claimed
+    // id is kept; a member with one stage more per pair reads ahead less far, so the ids it needs
+    // are there even earlier)
     const int ns_min = (base + kStageVecs - 1) / kStageVecs;
     const int ahead = 2 + (kRing - 2) / (ns_min > 0 ? ns_min : 1);
     if (tid == 0) {
-        for (int k = 0; k < ahead; ++k) sh.items[k] = cluster_id + k * n_clusters;
+        for (int k = 0; k < ahead; ++k) sh.items[k] = group_id + k * n_groups;
         for (int s = 0; s < kRing; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kStreamWarps); sh.armed[s] = 0; }
-        mbar_init(&sh.xbar[0], 1); mbar_init(&sh.xbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {
+    if (threadIdx.x < 32) {                          // one allocation for both virtual CTAs: all of the SM's columns
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&sh.tmem_base)), "r"(kTmemCols) : "memory");
+                     ::"r"(smem_u32(tmem_base_slot)), "r"(kStreamHalves * kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    cluster.sync();                                  // barriers of every CTA exist before any peer arrives on them
+    __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // warp w owns tensor-memory lanes 32*(w%4)..+31 and columns kTmemPerThread*(w/4)..
-    const uint32_t taddr = sh.tmem_base + (static_cast<uint32_t>(32 * (warp & 3)) << 16) + static_cast<uint32_t>(kTmemPerThread * (warp >> 2));
+    // warp w of a virtual CTA owns tensor-memory lanes 32*(w%4)..+31 and columns kTmemCols*half + kTmemPerThread*(w/4)..
+    const uint32_t taddr = *tmem_base_slot + (static_cast<uint32_t>(32 * (warp & 3)) << 16) +
+                           static_cast<uint32_t>(kTmemCols * half + kTmemPerThread * (warp >> 2));
+    // where this group's virtual CTAs exchange their statistics: [parity][rank] messages
+    GroupMsg* const xg = P.exchange + static_cast<size_t>(group_id < n_groups ? group_id : 0) * 2 * C;
 
     bool dead = false;                               // a bounded wait of this thread ran out
 
     // ---- producer: stage number -> (pair, slice part); any thread may issue a stage ----
-    // Stage gg of this CTA is part gg % ns of the (gg / ns)-th pair of this cluster (its id is in
+    // Stage gg of this virtual CTA is part gg % ns of the (gg / ns)-th pair of its group (its id is in
     // sh.items).  Stage gg + kRing is issued by the duty warp of stage gg + 1 (see the first sweep), so the
     // copies go out early and the work is spread over the warps.
     auto issue_stage = [&](uint32_t gg) {
@@ -397,27 +400,27 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
         bulk_g2s(dst, a_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
         bulk_g2s(dst + kStageRowBytes, b_row + (static_cast<size_t>(vbeg) + v0) * 16, bytes, &sh.full[slot]);
     };
-    if (tid == 0) {
+    if (tid == 0 && active) {
         for (uint32_t gg = 0; gg < kRing; ++gg) issue_stage(gg);
     }
     __syncwarp();
 
     float ereg[(NR > 0 ? NR : 1) * EPS];
     uint32_t g = 0;                                  // first ring stage of the current pair
-    uint32_t li = 0;                                 // pairs this cluster has finished
+    uint32_t li = 0;                                 // pairs this group has finished
     float x_carry = 0.f;                             // previous pair's second-sweep sum of this warp
     int prev_item = -1;                              // pair whose second-sweep sum is still to be published
-    int item = cluster_id;
+    int item = active ? group_id : P.n_items;
     uint32_t claimed = 0;                            // rank 0, combiner lane 0: the pair id taken this round
 
     for (;;) {
         const bool live = item < P.n_items;          // one extra round publishes the last pair's second sweep
         if (!live && prev_item < 0) break;
         const int par = static_cast<int>(li & 1);
-        const uint32_t xphase = (li >> 1) & 1;
+        const uint32_t tag = li + 1;                 // what this round's messages carry (never 0, the buffer's initial state)
         if (rank == 0 && lane == 0 && warp == static_cast<int>(li & (kStreamWarps - 1))) {
             // asked now, needed only when the statistics go out
-            const long long id = static_cast<long long>(ahead) * n_clusters + atomicAdd(P.next_pair, 1);
+            const long long id = static_cast<long long>(ahead) * n_groups + atomicAdd(P.next_pair, 1);
             claimed = id < 0x3fffffffLL ? static_cast<uint32_t>(id) : 0x3fffffffu;
         }
         bool bad = false;
@@ -613,16 +616,16 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
 
         // ---- exchange.  Every warp leaves its statistics in shared memory and counts itself in
         //      on a named barrier; this round's combiner warp waits there for the others, folds
-        //      the warps' statistics, sends the CTA's to every CTA of the cluster (itself
-        //      included), waits for all of the cluster's to land, folds those and leaves the
-        //      totals for the CTA.  Only the combiner polls; everyone else sleeps on a barrier. ----
+        //      the warps' statistics, stores the virtual CTA's message, fetches the group's messages
+        //      until all carry this round's tag, folds those and leaves the totals for the virtual
+        //      CTA.  Only the combiner polls; everyone else sleeps on a barrier. ----
         if (lane == 0) sh.ws[warp] = mine;
         __syncwarp();
         if (warp != static_cast<int>(li & (kStreamWarps - 1))) {
             __threadfence_block();
-            named_arrive(kBarPosted);
+            named_arrive(bar_posted);
         } else {
-            named_sync(kBarPosted);
+            named_sync(bar_posted);
             Stats w;
             w.ka = -INFINITY; w.kb = -INFINITY; w.za = 0.f; w.zb = 0.f; w.s0 = 0.f; w.sb = 0.f; w.x = 0.f; w.diff = 0;
             if (lane < kStreamWarps) w = sh.ws[lane];
@@ -647,17 +650,38 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
                 const uint32_t cl = __shfl_sync(0xffffffffu, claimed, 0);   // rank 0's message carries the pair id it took
                 if (rank == 0) c.diff |= cl << 1;
             }
-            if (lane == 0) mbar_arrive_expect_tx(&sh.xbar[par], static_cast<uint32_t>(C) * sizeof(Stats));
-            if (lane < C) {                                // lanes 0..15 hold the CTA's statistics; lane r serves CTA r
-                Stats* dst = &sh.xch[par][rank];
-                st_async_remote(dst, &sh.xbar[par], static_cast<uint32_t>(lane), c.ka, c.kb, c.za, c.zb);
-                st_async_remote(&dst->s0, &sh.xbar[par], static_cast<uint32_t>(lane), c.s0, c.sb, c.x, __uint_as_float(c.diff));
+            // lanes 0..2 each store one 16-byte unit of this virtual CTA's message; every unit ends in the round's tag
+            if (lane < 3) {
+                const float m0 = lane == 0 ? c.ka : lane == 1 ? c.zb : c.x;
+                const float m1 = lane == 0 ? c.kb : lane == 1 ? c.s0 : __uint_as_float(c.diff);
+                const float m2 = lane == 0 ? c.za : lane == 1 ? c.sb : 0.f;
+                st_unit(&xg[par * C + rank].u[lane], m0, m1, m2, tag);
             }
-            mbar_wait_cluster(&sh.xbar[par], xphase, P.timeout_flag, dead);
-            // cluster totals for the second sweep (float is enough there); lane r holds CTA r's part
+            // group totals for the second sweep (float is enough there); lane r fetches virtual CTA r's message
             Stats t;
             t.ka = -INFINITY; t.kb = -INFINITY; t.za = 0.f; t.zb = 0.f; t.s0 = 0.f; t.sb = 0.f; t.x = 0.f; t.diff = 0;
-            if (lane < C) t = sh.xch[par][lane];
+            if (!dead) {
+                bool got = false;
+#pragma unroll 1
+                for (uint32_t i = 0; i < kSpinLimit; ++i) {
+                    bool ok = true;
+                    if (lane < C) {
+                        const uint4 u0 = ld_unit(&xg[par * C + lane].u[0]), u1 = ld_unit(&xg[par * C + lane].u[1]),
+                                    u2 = ld_unit(&xg[par * C + lane].u[2]);
+                        ok = u0.w == tag && u1.w == tag && u2.w == tag;
+                        t.ka = __uint_as_float(u0.x); t.kb = __uint_as_float(u0.y); t.za = __uint_as_float(u0.z);
+                        t.zb = __uint_as_float(u1.x); t.s0 = __uint_as_float(u1.y); t.sb = __uint_as_float(u1.z);
+                        t.x = __uint_as_float(u2.x); t.diff = u2.y;
+                    }
+                    if (__all_sync(0xffffffffu, ok)) { got = true; break; }
+                    if ((i & 255u) == 255u && *reinterpret_cast<volatile int*>(P.timeout_flag) != 0) break;
+                }
+                if (!got) {
+                    if (lane == 0) atomicExch(P.timeout_flag, 1);
+                    dead = true;
+                    t.ka = __int_as_float(0x7fc00000);   // the totals of a round that never completed are invalid
+                }
+            }
             {
                 const uint32_t nxt = __shfl_sync(0xffffffffu, t.diff, 0) >> 1;
                 t.diff &= 1u;
@@ -671,20 +695,20 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
                 tza += __shfl_xor_sync(0xffffffffu, tza, m); tzb += __shfl_xor_sync(0xffffffffu, tzb, m);
             }
             if (lane == 0) *reinterpret_cast<float4*>(sh.tot) = make_float4(Ka, Kb, tza, tzb);
-            named_sync(kBarTotals);
+            named_sync(bar_totals);
             // rank 0 hands the parts to the finish kernel, which folds them in double; the
             // previous pair gets its second-sweep sums
             if (rank == 0 && lane < C) {
                 if (prev_item >= 0) P.records[prev_item].x[lane] = t.x;
                 if (live) {
-                    FSD_CHECK(P.timeout_flag + 2, item >= 0 && item < P.n_items && C <= kStreamMaxCluster, kChkRecord);
+                    FSD_CHECK(P.timeout_flag + 2, item >= 0 && item < P.n_items && C <= kMaxGroupSize, kChkRecord);
                     PairRecord* r = P.records + item;
                     r->part[lane] = t;
                     if (lane == 0) { r->ncta = static_cast<uint32_t>(C); r->state = bad ? kRecordBadTree : kRecordStats; }
                 }
             }
         }
-        if (warp != static_cast<int>(li & (kStreamWarps - 1))) named_sync(kBarTotals);
+        if (warp != static_cast<int>(li & (kStreamWarps - 1))) named_sync(bar_totals);
         const float4 tot = *reinterpret_cast<const float4*>(sh.tot);
         const float Ka = tot.x, Kb = tot.y, tZa = tot.z, tZb = tot.w;
         prev_item = -1;
@@ -754,7 +778,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (tid == 0) {
-        // Every copy started into this CTA's ring has landed before the CTA may leave: normally the
+        // Every copy started into this virtual CTA's ring has landed before the CTA may leave: normally the
         // first sweep consumed them all and these waits return at once; after a wait that ran out
         // some may still be on their way (a copy, once started, always completes).
         for (int slot = 0; slot < kRing; ++slot) {
@@ -766,20 +790,9 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_pair_str
         }
     }
     __syncthreads();
-    if (warp == 0) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sh.tmem_base), "r"(kTmemCols) : "memory");
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_base_slot), "r"(kStreamHalves * kTmemCols) : "memory");
     }
-    cluster.sync();                                    // nobody leaves while a peer may still write to or read from it
-}
-
-// Occupancy twin: same block size, register bound and dynamic shared memory as the streaming
-// kernel but no tensor-memory instructions.  The occupancy calculator assumes one resident CTA
-// per SM for any kernel that allocates tensor memory (it cannot know how many columns); the
-// streaming kernel allocates half of an SM's tensor memory, so two CTAs do fit, and the grid
-// is sized from this twin instead.
-__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) fsd_stream_occupancy_twin(int* p) {
-    extern __shared__ unsigned char smem_raw[];
-    if (p != nullptr) p[threadIdx.x] = smem_raw[threadIdx.x];
 }
 
 }  // namespace fsd

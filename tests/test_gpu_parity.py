@@ -81,10 +81,10 @@ def test_paper_candidate_lengths_at_a_full_vocabulary(gamma):
 
 
 @pytest.mark.parametrize("dtype,V", [("bf16", 32776), ("f32", 16388), ("bf16", 65544), ("bf16", 131080)])
-def test_slices_of_unequal_stage_counts_within_a_cluster(dtype, V):
-    """Row lengths that split over the cluster into slices of which some need one ring stage more
-    than the others, with more pairs than the clusters take in their first rounds: the CTAs of a
-    cluster must still agree on which pair comes next."""
+def test_slices_of_unequal_stage_counts_within_a_group(dtype, V):
+    """Row lengths that split over a group of virtual CTAs into slices of which some need one ring
+    stage more than the others, with more pairs than the groups take in their first rounds: the
+    members of a group must still agree on which pair comes next."""
     c = gi.make_chain(16, 8, V, dtype=dtype, recipe="zipf", sigma=(0.2, 1.5), sigma_mode="uniform",
                       disjoint_frac=0.1, workload_id=420)
     r = _check(c, T=0.2)
@@ -212,9 +212,9 @@ def test_fsd_outputs_do_not_depend_on_tokens_or_accept_uniforms():
 
 
 @pytest.mark.parametrize("dtype,V", [("f32", 100000), ("f32", 152064), ("bf16", 200008), ("bf16", 256000)])
-def test_vocabularies_that_need_sixteen_cta_clusters(dtype, V):
-    """Rows too long for eight CTAs' on-chip capacity (fp32 above 81920 entries, bf16 above
-    163840) are streamed by clusters of sixteen."""
+def test_vocabularies_that_need_groups_of_more_than_eight(dtype, V):
+    """Rows too long for eight virtual CTAs' on-chip capacity (fp32 above 81920 entries, bf16 above
+    163840) are streamed by larger groups (up to sixteen)."""
     c = gi.make_chain(5, 4, V, dtype=dtype, recipe="zipf", sigma=(0.3, 1.5), sigma_mode="uniform",
                       disjoint_frac=0.1, workload_id=309)
     for div in ("js", "kl", "tv"):

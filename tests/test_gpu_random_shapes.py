@@ -1,7 +1,7 @@
 """GPU-vs-oracle parity on seeded random shapes, dtypes, divergences, modes and thresholds.
 
 The named workloads fix a handful of shapes; this sweep draws others (vocabulary sizes that are
-and are not multiples of the vector width, cluster sizes 1 to 8, one to five ring stages per
+and are not multiples of the vector width, group sizes 1 to 16, one to five ring stages per
 pair, masked entries) so that every launch configuration of the pair kernels meets the oracle.
 """
 
