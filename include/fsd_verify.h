@@ -216,6 +216,16 @@ int fsd_set_stage_event(void *event);
  * Process-wide, read when a call is made; off by default.  Returns FSD_OK. */
 int fsd_set_timeout_injection(int on);
 
+/* Test and tuning aid (no counterpart in the paper).  The streaming kernel splits every
+ * (row, position) pair along the vocabulary over a group of 1..16 thread blocks; the library
+ * picks the group size from the row length and the number of pairs.  A nonzero `group_size`
+ * replaces that choice in later verify calls wherever it is possible (at least the smallest
+ * size whose slice fits on chip, at most 16; otherwise the library's own choice stands); 0
+ * restores the library's choice.  Results do not depend on the group size beyond the order of
+ * floating-point additions.  Process-wide, read when a call is made.  Returns FSD_OK, or
+ * FSD_ERR_SHAPE for a size outside 0..16. */
+int fsd_set_group_size(int group_size);
+
 /* Debug build (no counterpart in the paper).  A library compiled with -DFSD_DEBUG_CHECKS
  * (python -m paper_2502_20704_b200.build --debug) checks, inside its kernels, the indices and
  * ranges behind its memory accesses -- pair ids, slice and stage bounds of the copies, tensor-

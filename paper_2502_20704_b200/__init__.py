@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     fsd_default_opts,
     fsd_host_staging_bytes,
     fsd_set_stage_event,
+    fsd_set_group_size,
     fsd_set_timeout_injection,
     fsd_status_string,
     fsd_threshold_sweep,

@@ -90,6 +90,8 @@ def _load():
         lib.fsd_debug_checks.restype = C.c_int
         lib.fsd_set_timeout_injection.argtypes = [C.c_int]
         lib.fsd_set_timeout_injection.restype = C.c_int
+        lib.fsd_set_group_size.argtypes = [C.c_int]
+        lib.fsd_set_group_size.restype = C.c_int
         lib.fsd_threshold_sweep.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, C.c_int, vp, vp, C.c_void_p]
         lib.fsd_threshold_sweep.restype = C.c_int
         lib.fsd_calibrate_threshold.argtypes = [vp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, C.c_void_p]
@@ -150,6 +152,12 @@ def fsd_set_timeout_injection(on: bool) -> int:
     """While on, verify calls report FSD_ROW_TIMEOUT in every row as if a bounded device-side wait
     had run out (a test aid; off by default)."""
     return _load().fsd_set_timeout_injection(1 if on else 0)
+
+
+def fsd_set_group_size(group_size: int) -> int:
+    """Thread blocks a pair is split over in the streaming kernel (a test and tuning aid); 0: the
+    library chooses."""
+    return _load().fsd_set_group_size(int(group_size))
 
 
 def fsd_workspace_bytes(B: int, positions: int, V: int, opts: FsdOpts) -> int:

@@ -80,6 +80,7 @@ int finish_cluster_size(int B, int V) {
 
 std::atomic<void*> g_stage_event{nullptr};   // see fsd_set_stage_event
 std::atomic<int> g_mark_timeout{0};          // see fsd_set_timeout_injection
+std::atomic<int> g_group_size{0};            // see fsd_set_group_size
 
 // ---- streaming kernel launch -----------------------------------------------------------
 constexpr int kMaxDev = 64;
@@ -134,6 +135,8 @@ int launch_stream(const StreamParams& gp, int nsm, cudaStream_t s) {
 int group_size(int nvec_row, bool vec, int items, int nsm) {
     if (!vec || nvec_row < 64) return 0;
     const int cmin = (nvec_row + kMaxVecPerCta - 1) / kMaxVecPerCta;
+    const int forced = g_group_size.load();
+    if (forced >= cmin && forced <= kMaxGroupSize && cmin <= kMaxGroupSize) return forced;
     int vctas = kStreamHalves * nsm;
     if (vctas > kMaxVirtualCtas) vctas = kMaxVirtualCtas;
     int best = 0;
@@ -466,6 +469,12 @@ int fsd_debug_checks(int B, int positions, size_t* word_offset) {
 
 int fsd_set_timeout_injection(int on) {
     g_mark_timeout.store(on != 0 ? 1 : 0);
+    return FSD_OK;
+}
+
+int fsd_set_group_size(int group_size) {
+    if (group_size < 0 || group_size > kMaxGroupSize) return FSD_ERR_SHAPE;
+    g_group_size.store(group_size);
     return FSD_OK;
 }
 

@@ -60,8 +60,9 @@ struct FinishShared {
     FinishExchange slot;
     FinishExchange all[kMaxClusterSize];   // what the cluster's CTAs published (see cluster_exchange)
     double sc[kMaxClusterSize];
-    double gather_d[kMaxClusterSize];   // one value per CTA of the cluster (see cluster_gather)
-    int gather_i[kMaxClusterSize];
+    double gather_d[2][kMaxClusterSize];   // one value per CTA of the cluster, written by the peers (see cluster_gather)
+    int gather_i[2][kMaxClusterSize];
+    float kref[kMaxTreeNodes];          // per pair: integer reference at or just above the target row's log2-sum-exp (NaN: none)
     double exp_table[kExpTable];   // 2^(j/256)
     double red_d[32 * 2];
     float red_f[32 * 2];
@@ -108,15 +109,17 @@ __device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Fin
     cluster.sync();
 }
 
-// Light exchange: every CTA publishes one double and one int; afterwards sh.gather_d / gather_i
-// hold the values of all CTAs, in rank order, in every CTA.  Two cluster barriers.
-__device__ __forceinline__ void cluster_gather(cg::cluster_group& cluster, FinishShared& sh, int cs, double v, int iv) {
-    if (threadIdx.x == 0) { sh.slot.d[0] = v; sh.slot.i[0] = iv; }
-    cluster.sync();
+// Light exchange: every CTA writes one double and one int into every CTA's shared memory (its
+// own included); after ONE cluster barrier sh.gather_d[buf] / gather_i[buf] hold the values of
+// all CTAs, in rank order, in every CTA, and nobody reads a peer's memory (so a CTA may leave
+// right afterwards).  `buf` alternates from one call to the next: a CTA that is already writing
+// the next exchange cannot disturb the values a slower peer is still reading.  The peers must be
+// known to have started (one cluster barrier earlier in the kernel).
+__device__ __forceinline__ void cluster_gather(cg::cluster_group& cluster, FinishShared& sh, int cs, int rank, int buf, double v, int iv) {
     if (threadIdx.x < cs) {
-        const FinishShared* rs = cluster.map_shared_rank(&sh, threadIdx.x);
-        sh.gather_d[threadIdx.x] = rs->slot.d[0];
-        sh.gather_i[threadIdx.x] = rs->slot.i[0];
+        FinishShared* rs = cluster.map_shared_rank(&sh, threadIdx.x);
+        rs->gather_d[buf][rank] = v;
+        rs->gather_i[buf][rank] = iv;
     }
     cluster.sync();
 }
@@ -129,6 +132,7 @@ struct PairTotals {
     double Za, Zb, Sa, Sb, K, X;
     float ka, kb;
     uint32_t differ;
+    uint32_t state;            // the record's state word
 };
 // 2^d for an integer-valued d <= 0, exact; 0 below the normal range
 __device__ __forceinline__ double pow2_int_d(double d) {
@@ -144,10 +148,17 @@ __device__ __forceinline__ double group_sum(double v) {       // over the kMaxGr
 __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     const int r = threadIdx.x & (kMaxGroupSize - 1);
     PairTotals t;
+    t.state = 0;
     Stats c;
     c.ka = -INFINITY; c.kb = -INFINITY; c.za = 0.f; c.zb = 0.f; c.s0 = 0.f; c.sb = 0.f; c.x = 0.f; c.diff = 0;
     float x = 0.f;
-    if (rec != nullptr && r < static_cast<int>(rec->ncta)) { c = rec->part[r]; x = rec->x[r]; }
+    if (rec != nullptr) {
+        // every lane fetches its part at once with the count (one trip to L2); parts beyond the count are stale
+        const Stats cr = rec->part[r];
+        const float xr = rec->x[r];
+        t.state = rec->state;
+        if (r < static_cast<int>(rec->ncta)) { c = cr; x = xr; }
+    }
     float ka = c.ka, kb = c.kb;                          // NaN references win
 #pragma unroll
     for (int m = kMaxGroupSize / 2; m > 0; m >>= 1) {
@@ -180,15 +191,15 @@ __device__ inline PairTotals fold_record(const PairRecord* rec, int div) {
     return t;
 }
 
-__device__ inline void judge_record(const FinishParams& P, int item, const PairTotals& r, const void* a_row, const void* b_row, int dt,
-                                    float& D_out, int& bit_out, int& st_out) {
-    if (P.records[item].state & kRecordBadTree) {
+__device__ inline void judge_record(const FinishParams& P, int item, const PairTotals& r, double lnZa, double lnZb,
+                                    const void* a_row, const void* b_row, int dt, float& D_out, int& bit_out, int& st_out) {
+    if (r.state & kRecordBadTree) {
         D_out = __int_as_float(0x7fc00000); bit_out = 0; st_out = FSD_ROW_BADTREE;
         return;
     }
     const bool finite = isfinite(r.ka) && isfinite(r.kb) && r.Za > 0.0 && r.Zb > 0.0 && isfinite(r.Za) && isfinite(r.Zb);
     float D = __int_as_float(0x7fc00000);
-    if (finite) D = r.differ ? static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, r.Sa, r.Sb, r.K, r.X)) : 0.0f;
+    if (finite) D = r.differ ? static_cast<float>(combine_divergence(P.div, r.Za, r.Zb, lnZa, lnZb, r.Sa, r.Sb, r.K, r.X)) : 0.0f;
     const bool div_ok = finite && passes(D, P.T, P.cmp);
     int bit = div_ok;
     if (P.mode != FSD_MODE_FSD) {
@@ -203,8 +214,8 @@ __device__ inline void judge_record(const FinishParams& P, int item, const PairT
                     pacc = (ax != -INFINITY) ? 1.0 : 0.0;
                 } else {
                     // ln P(x) = (x*log2e - k) ln2 - ln Z with the same float log2e the sums were built with
-                    const double la = (static_cast<double>(ax) * static_cast<double>(kLog2e) - r.ka) * kLn2D - log(r.Za);
-                    const double lb = (static_cast<double>(bx) * static_cast<double>(kLog2e) - r.kb) * kLn2D - log(r.Zb);
+                    const double la = (static_cast<double>(ax) * static_cast<double>(kLog2e) - r.ka) * kLn2D - lnZa;
+                    const double lb = (static_cast<double>(bx) * static_cast<double>(kLog2e) - r.kb) * kLn2D - lnZb;
                     pacc = exp(la - lb);
                     pacc = pacc < 1.0 ? pacc : 1.0;
                 }
@@ -320,20 +331,27 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const char* d_base = static_cast<const char*>(P.draft) + static_cast<size_t>(b) * G * rb;
     const bool tree = P.parent != nullptr;
 
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");     // "this CTA has started": waited for below
     if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; sh.token = -1; }
-    if (tid < kExpTable) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / kExpTable));
     __syncthreads();
     // everything above touched no global memory; what follows reads what the pair kernel wrote
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");       // every CTA of the cluster runs: its shared memory may be written
 
     // ---- 1. divergences, accept bits, status of this row's pairs ----
+    // (asked for now, needed later: each is a trip to L2 or HBM of its own)
+    const float u_draw = P.u_sample[b];
     int st = 0, first = G;
+    if (tid == 0 && P.timeout_flag != nullptr && *reinterpret_cast<const volatile int*>(P.timeout_flag) != 0) st |= FSD_ROW_TIMEOUT;
     if (P.records != nullptr) {
         // two pairs per warp: sixteen lanes fold a pair's record, the first of them judges it
         for (int i0 = 2 * warp; i0 < G; i0 += 2 * (blockDim.x >> 5)) {
             const int i = i0 + (lane >> 4);
             const int item = b * G + i;
             const PairTotals tot = fold_record(i < G ? P.records + item : nullptr, P.div);
+            // the two logarithms the judgement needs, by two lanes at once
+            const double lz = log((lane & 15) == 1 ? tot.Zb : tot.Za);
+            const double lnZa = lz, lnZb = __shfl_down_sync(0xffffffffu, lz, 1);
             if (i < G && (lane & 15) == 0) {
                 int trow = i;
                 if (tree) {
@@ -342,9 +360,14 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                 }
                 float D;
                 int bit, s;
-                judge_record(P, item, tot, t_base + static_cast<size_t>(trow) * rb, d_base + static_cast<size_t>(i) * rb, DT, D, bit, s);
+                judge_record(P, item, tot, lnZa, lnZb, t_base + static_cast<size_t>(trow) * rb, d_base + static_cast<size_t>(i) * rb, DT, D, bit, s);
                 if (rank == 0) P.divergence[item] = D;
                 st |= s;
+                if (i < kMaxTreeNodes) {
+                    const float za = static_cast<float>(tot.Za);
+                    const bool ok = s == 0 && isfinite(tot.ka) && za > 0.f && za < 3.0e38f;
+                    sh.kref[i] = ok ? ceilf(tot.ka + log2f(za)) : __int_as_float(0x7fc00000);
+                }
                 if (tree) sh.tree_bit[i] = static_cast<int8_t>(bit);
                 else if (!bit && i < first) first = i;
             }
@@ -358,7 +381,6 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             else if (!bit && i < first) first = i;
         }
     }
-    if (tid == 0 && P.timeout_flag != nullptr && *P.timeout_flag != 0) st |= FSD_ROW_TIMEOUT;
     st = __reduce_or_sync(0xffffffffu, st);
     first = __reduce_min_sync(0xffffffffu, first);
     if (lane == 0) {
@@ -414,33 +436,17 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         // row maximum.
         float kref = 0.f;
         bool have_ref = false;
-        if (P.records != nullptr && !tree && n < G) {
-            const PairRecord* r = P.records + (static_cast<size_t>(b) * G + n);
-            if (r->state & kRecordStats) {
-                float rka = -INFINITY;
-                bool nan = false;
-                for (uint32_t c = 0; c < r->ncta && c < kMaxGroupSize; ++c) {
-                    const float a = r->part[c].ka;
-                    nan = nan || a != a;
-                    rka = fmaxf(rka, a);
-                }
-                if (!nan && isfinite(rka)) {
-                    float za = 0.f;
-                    for (uint32_t c = 0; c < r->ncta && c < kMaxGroupSize; ++c) {
-                        const float a = r->part[c].ka;
-                        if (a != -INFINITY) za += r->part[c].za * pow2_int(a - rka);
-                    }
-                    if (za > 0.f && za < 3.0e38f) { kref = ceilf(rka + log2f(za)); have_ref = true; }
-                }
-            }
+        if (P.records != nullptr && !tree && n < G && n < kMaxTreeNodes) {
+            kref = sh.kref[n];                            // left by the thread that judged the rejected pair
+            have_ref = kref == kref;
         }
         if (!have_ref) {
             float m[1] = {-INFINITY};
             for_chunk<DT>(a_row, b_row, k0, k1, vec, false, [&](int, float xa, float) { m[0] = fmaxf(m[0], xa); });
             block_max<1>(m, sh.red_f);
-            cluster_gather(cluster, sh, cs, m[0], 0);
+            cluster_gather(cluster, sh, cs, rank, 0, m[0], 0);
             double M = -INFINITY;
-            for (int r = 0; r < cs; ++r) M = fmax(M, sh.gather_d[r]);
+            for (int r = 0; r < cs; ++r) M = fmax(M, sh.gather_d[0][r]);
             if (!isfinite(M)) {                           // no finite logit, or +inf: uniform over the cluster
                 if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.next_token[b] = -1; P.row_status[b] = status | FSD_ROW_NONFINITE; }
                 return;
@@ -470,20 +476,20 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         }
         incl += wpre;
         excl += wpre;
-        cluster_gather(cluster, sh, cs, cta_tot, 0);
+        cluster_gather(cluster, sh, cs, rank, 1, cta_tot, 0);
         double W = 0.0;
-        for (int r = 0; r < cs; ++r) W += sh.gather_d[r];
+        for (int r = 0; r < cs; ++r) W += sh.gather_d[1][r];
         if (!(isfinite(W) && W > 0.0)) {                  // NaN logit (or nothing representable): uniform over the cluster
             if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.next_token[b] = -1; P.row_status[b] = status | FSD_ROW_NONFINITE; }
             return;
         }
         if (rank == 0 && tid == 0) { P.accept_len[b] = n; P.row_status[b] = status; }
-        const double t = static_cast<double>(P.u_sample[b]) * W;
+        const double t = static_cast<double>(u_draw) * W;
         double cpre = 0.0, run = 0.0;
         int owner = -1;
         for (int r = 0; r < cs && owner < 0; ++r) {
             cpre = run;
-            run += sh.gather_d[r];
+            run += sh.gather_d[1][r];
             if (run > t) owner = r;
         }
         auto last_with_weight = [&]() -> int {           // highest index of this thread's chunk whose weight is positive
@@ -495,9 +501,9 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             const int lp = __reduce_max_sync(0xffffffffu, last_with_weight());
             if (lane == 0 && lp >= 0) atomicMax(&sh.last_pos, lp);
             __syncthreads();
-            cluster_gather(cluster, sh, cs, 0.0, sh.last_pos);
+            cluster_gather(cluster, sh, cs, rank, 0, 0.0, sh.last_pos);
             int best = -1;
-            for (int r = 0; r < cs; ++r) best = sh.gather_i[r] > best ? sh.gather_i[r] : best;
+            for (int r = 0; r < cs; ++r) best = sh.gather_i[0][r] > best ? sh.gather_i[0][r] : best;
             if (rank == 0 && tid == 0) P.next_token[b] = best;
             return;
         }
@@ -512,34 +518,72 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             __syncthreads();
             if (tid == 0) P.next_token[b] = sh.last_pos;
         } else if (warp == (c >> 5)) {
-            // the warp of the thread whose chunk holds the crossing walks that chunk together:
-            // 32 weights at a time, prefix sums in index order
+            // The warp of the thread whose chunk holds the crossing walks that chunk together: lane j
+            // takes the chunk's j-th unit (a 16-byte vector, or one entry of an unaligned row) and sums
+            // its weights in index order; every lane then adds the units' sums in order until the
+            // running sum passes the target, and the lane of that unit finds the entry.
             const int src = c & 31;
             const int ck0 = __shfl_sync(0xffffffffu, k0, src), ck1 = __shfl_sync(0xffffffffu, k1, src);
-            double base = __shfl_sync(0xffffffffu, excl, src);
-            int tok = 0x7fffffff, lastp = -1;
-            for (int kb = ck0; kb < ck1; kb += 32) {
-                const int k = kb + lane;
-                double w = 0.0;
-                if (k < ck1) w = static_cast<double>(weight(load_logit<DT>(a_row, k)));
-                double run = w;
+            double run = __shfl_sync(0xffffffffu, excl, src);
+            const int U = vec ? EPV : 1;
+            int tok = -1, lastp = -1;
+            for (int u0 = ck0; u0 < ck1 && tok < 0; u0 += 32 * U) {
+                const int uk = u0 + lane * U;
+                float w[EPV];
 #pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const double up = __shfl_up_sync(0xffffffffu, run, d);
-                    if (lane >= d) run += up;
+                for (int j = 0; j < EPV; ++j) w[j] = 0.f;
+                if (uk < ck1) {
+                    if (vec) {
+                        float xa[EPV];
+                        unpack_vec<DT>(ldg_vec(a_row, uk / EPV), xa);
+#pragma unroll
+                        for (int j = 0; j < EPV; ++j) w[j] = weight(xa[j]);
+                    } else {
+                        w[0] = weight(load_logit<DT>(a_row, uk));
+                    }
                 }
-                run += base;
-                if (w > 0.0) lastp = k;
-                if (w > 0.0 && run > t_local && k < tok) tok = k;
-                base = __shfl_sync(0xffffffffu, run, 31);
+                double usum = 0.0;
+                int ulast = -1;
+#pragma unroll
+                for (int j = 0; j < EPV; ++j) {
+                    usum += static_cast<double>(w[j]);
+                    if (w[j] > 0.f) ulast = uk + j;
+                }
+                int hit = -1;                            // unit in which the running sum passes the target
+                double before = 0.0;                     // the running sum in front of that unit
+                const int nunits = min(32, (ck1 - u0 + U - 1) / U);
+                for (int j = 0; j < nunits; ++j) {
+                    const double sj = __shfl_sync(0xffffffffu, usum, j);
+                    if (hit < 0) {
+                        if (sj > 0.0 && run + sj > t_local) { hit = j; before = run; }
+                        else run += sj;
+                    }
+                }
+                lastp = max(lastp, __reduce_max_sync(0xffffffffu, ulast));
+                if (hit >= 0) {
+                    int t_here = -1;
+                    if (lane == hit) {
+                        double r2 = before;
+#pragma unroll
+                        for (int j = 0; j < EPV; ++j) {
+                            r2 += static_cast<double>(w[j]);
+                            if (t_here < 0 && w[j] > 0.f && r2 > t_local) t_here = uk + j;
+                        }
+                        if (t_here < 0) t_here = ulast;   // lost to the order of the additions: the unit's last entry with weight
+                    }
+                    tok = __shfl_sync(0xffffffffu, t_here, hit);
+                }
             }
-            tok = __reduce_min_sync(0xffffffffu, tok);
-            lastp = __reduce_max_sync(0xffffffffu, lastp);
-            FSD_CHECK(P.debug_word, (tok != 0x7fffffff ? tok : lastp) >= -1 && (tok != 0x7fffffff ? tok : lastp) < V, kChkToken);
-            if (lane == 0) P.next_token[b] = tok != 0x7fffffff ? tok : lastp;
+            if (tok < 0) tok = lastp;
+            FSD_CHECK(P.debug_word, tok >= -1 && tok < V, kChkToken);
+            if (lane == 0) P.next_token[b] = tok;
         }
         return;
     }
+
+    // the paths below take their exponentials in double precision from a table
+    if (tid < kExpTable) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / kExpTable));
+    __syncthreads();
 
     // ---- references.  A residual draw follows a rejection, so the rejected pair's record has
     //      references (log2 domain) for both rows, near their maxima and common to the cluster;
@@ -738,7 +782,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             return;
         }
 
-        const double t = static_cast<double>(P.u_sample[b]) * W;
+        const double t = static_cast<double>(u_draw) * W;
         double cpre = 0.0, run = 0.0;
         int owner = -1, last_any = -1;
         for (int r = 0; r < cs; ++r) {

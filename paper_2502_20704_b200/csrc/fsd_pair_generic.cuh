@@ -32,8 +32,8 @@ struct PairParams {
 //   K        sum_k 2^(ya_k) * (ya_k - yb_k)             (KL, Appendix C.1)
 //   X        JS: sum_k s_k log2 s_k with s = p + q;  TV: sum_k |p_k - q_k|
 // Returns the divergence in nats (NaN when a row is not a valid distribution).
-__device__ inline double combine_divergence(int div, double Za, double Zb, double Sa, double Sb, double K, double X) {
-    const double lnZa = log(Za), lnZb = log(Zb);
+// The variant with lnZa, lnZb takes the two logarithms from the caller (computed by two lanes at once).
+__device__ inline double combine_divergence(int div, double Za, double Zb, double lnZa, double lnZb, double Sa, double Sb, double K, double X) {
     double D;
     if (div == FSD_DIV_KL) {
         D = kLn2D * K / Za - lnZa + lnZb;
@@ -46,6 +46,9 @@ __device__ inline double combine_divergence(int div, double Za, double Zb, doubl
         D = 0.5 * X;
     }
     return D < 0.0 ? 0.0 : D;   // NaN stays NaN
+}
+__device__ inline double combine_divergence(int div, double Za, double Zb, double Sa, double Sb, double K, double X) {
+    return combine_divergence(div, Za, Zb, log(Za), log(Zb), Sa, Sb, K, X);
 }
 
 // ln P(x) of one token from its logit and the row's normaliser, in double.

@@ -222,6 +222,32 @@ def test_vocabularies_that_need_groups_of_more_than_eight(dtype, V):
     _check(c, mode="rfsd", T=0.25)
 
 
+@pytest.mark.parametrize("V,sizes", [(4096, (1, 2, 3, 5, 16)), (32000, (2, 3, 7, 11, 16)), (152064, (8, 9, 13, 16))])
+def test_every_group_size_gives_the_same_answers(V, sizes):
+    """The streaming kernel splits a pair over a group of thread blocks whose size the library
+    chooses; forced to other sizes (slices of one to five ring stages, even and uneven splits,
+    more and fewer groups than pairs) the kernel must agree with the oracle all the same, and
+    decisions and tokens must not depend on the size."""
+    from paper_2502_20704_b200 import binding as fsd
+
+    c = gi.make_chain(6, 5, V, dtype="bf16", recipe="zipf", sigma=(0.2, 1.5), sigma_mode="uniform",
+                      disjoint_frac=0.1, workload_id=430)
+    base = _check(c, T=0.2)["gpu"]
+    try:
+        for size in sizes:
+            assert fsd.fsd_set_group_size(size) == 0
+            for div in ("js", "kl", "tv"):
+                _check(c, div=div, T=0.2)
+            r = _check(c, T=0.2)["gpu"]
+            assert np.allclose(r.divergence, base.divergence, rtol=0, atol=2e-6)
+            clear = (np.abs(base.divergence - 0.2) > 1e-5).all(axis=1)      # rows with no divergence at the threshold
+            assert np.array_equal(r.accept_len[clear], base.accept_len[clear])
+            assert np.array_equal(r.next_token[clear], base.next_token[clear])
+    finally:
+        fsd.fsd_set_group_size(0)
+    assert fsd.fsd_set_group_size(17) != 0 and fsd.fsd_set_group_size(-1) != 0
+
+
 def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
     """Two workloads verified at once on two streams (separate workspaces, as the header asks):
     each must give exactly what it gives alone; a workspace reused call after call must, too."""
