@@ -209,12 +209,16 @@ int fsd_version(void);
 int fsd_set_stage_event(void *event);
 
 /* Test aid (no counterpart in the paper).  Every wait inside the streaming kernel is bounded; a
- * wait that runs out raises a flag in the workspace, the call still returns, and every row's
- * row_status carries FSD_ROW_TIMEOUT (its other outputs are then not valid).  While injection is
- * on, verify calls raise that flag themselves (a 4-byte memset between the two kernels), so the
- * reporting path can be exercised without making a GPU wait for something that never comes.
- * Process-wide, read when a call is made; off by default.  Returns FSD_OK. */
-int fsd_set_timeout_injection(int on);
+ * wait that runs out raises a flag in the workspace, the thread blocks that see it take no
+ * further work, the call still returns, and every row's row_status carries FSD_ROW_TIMEOUT (its
+ * other outputs are then not valid).  mode 1: verify calls raise that flag themselves (a 4-byte
+ * memset between the two kernels), which exercises the reporting path alone.  mode 2: in the
+ * streaming kernel one thread block keeps its first statistics message to itself and the limit
+ * of the exchange wait is lowered to about a tenth of a second, so its partners' wait really
+ * runs out and the kernel's own give-up path runs (every wait stays bounded; nothing faults).
+ * mode 0: off (the default).  Process-wide, read when a call is made.  Returns FSD_OK, or
+ * FSD_ERR_ENUM for another mode. */
+int fsd_set_timeout_injection(int mode);
 
 /* Test and tuning aid (no counterpart in the paper).  The streaming kernel splits every
  * (row, position) pair along the vocabulary over a group of 1..16 thread blocks; the library

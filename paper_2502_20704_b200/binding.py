@@ -148,10 +148,11 @@ def fsd_debug_checks(B: int = 0, positions: int = 0):
     return bool(on), (off.value if B >= 1 and positions >= 1 else None)
 
 
-def fsd_set_timeout_injection(on: bool) -> int:
-    """While on, verify calls report FSD_ROW_TIMEOUT in every row as if a bounded device-side wait
-    had run out (a test aid; off by default)."""
-    return _load().fsd_set_timeout_injection(1 if on else 0)
+def fsd_set_timeout_injection(mode) -> int:
+    """Test aid.  1 (or True): verify calls report FSD_ROW_TIMEOUT in every row as if a bounded
+    device-side wait had run out.  2: one thread block of the streaming kernel withholds a message,
+    so that a (shortened) device-side wait really runs out.  0 (or False): off."""
+    return _load().fsd_set_timeout_injection(int(mode))
 
 
 def fsd_set_group_size(group_size: int) -> int:

@@ -166,6 +166,11 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Grou
         sp.target = pp.target; sp.draft = pp.draft; sp.parent = pp.parent; sp.B = pp.B; sp.G = pp.G;
         sp.nvec_row = nvec_row; sp.n_items = items; sp.records = records; sp.timeout_flag = flags; sp.next_pair = flags + 1;
         sp.C = C; sp.exchange = exchange;
+        // test aid: one virtual CTA keeps its first message to itself, so that its group's exchange
+        // runs out (after a shorter limit: about a tenth of a second) and the kernel's own give-up path runs
+        const bool silent = g_mark_timeout.load() == 2;
+        sp.poll_limit = silent ? (1u << 17) : kSpinLimit;
+        sp.silent_rank = silent ? C - 1 : -1;
         // everything that can fail without a launch (attributes, the occupancy query) comes before
         // the first thing put on the stream
         int rc;
@@ -180,7 +185,7 @@ int launch_all(const PairParams& pp, FinishParams fp, bool vec, int* flags, Grou
         else                           rc = launch_stream<DT, FSD_DIV_TV>(sp, nsm, s);
         if (rc != FSD_OK) return rc;
         // test aid: behave as if a bounded wait of the streaming kernel had run out
-        if (g_mark_timeout.load() != 0 && cudaMemsetAsync(flags, 1, sizeof(int), s) != cudaSuccess) return FSD_ERR_CUDA;
+        if (g_mark_timeout.load() == 1 && cudaMemsetAsync(flags, 1, sizeof(int), s) != cudaSuccess) return FSD_ERR_CUDA;
         fp.timeout_flag = flags;
         fp.records = records;
     } else {
@@ -467,8 +472,9 @@ int fsd_debug_checks(int B, int positions, size_t* word_offset) {
 #endif
 }
 
-int fsd_set_timeout_injection(int on) {
-    g_mark_timeout.store(on != 0 ? 1 : 0);
+int fsd_set_timeout_injection(int mode) {
+    if (mode < 0 || mode > 2) return FSD_ERR_ENUM;
+    g_mark_timeout.store(mode);
     return FSD_OK;
 }
 

@@ -100,6 +100,8 @@ struct StreamParams {
     int* timeout_flag;         // set to 1 if a bounded wait ran out; zero at launch
     int* next_pair;            // pairs handed out beyond each group's fixed first ones; zero at launch
     int C;                     // virtual CTAs per group (<= kMaxGroupSize)
+    uint32_t poll_limit;       // fetches of the group's messages before the exchange gives up (kSpinLimit normally)
+    int silent_rank;           // test aid: this rank of group 0 keeps its first message to itself (-1: nobody)
     GroupMsg* exchange;        // [groups][2][C], zero at launch
 };
 
@@ -651,7 +653,7 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
                 if (rank == 0) c.diff |= cl << 1;
             }
             // lanes 0..2 each store one 16-byte unit of this virtual CTA's message; every unit ends in the round's tag
-            if (lane < 3) {
+            if (lane < 3 && !(li == 0 && group_id == 0 && rank == P.silent_rank)) {
                 const float m0 = lane == 0 ? c.ka : lane == 1 ? c.zb : c.x;
                 const float m1 = lane == 0 ? c.kb : lane == 1 ? c.s0 : __uint_as_float(c.diff);
                 const float m2 = lane == 0 ? c.za : lane == 1 ? c.sb : 0.f;
@@ -660,10 +662,15 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
             // group totals for the second sweep (float is enough there); lane r fetches virtual CTA r's message
             Stats t;
             t.ka = -INFINITY; t.kb = -INFINITY; t.za = 0.f; t.zb = 0.f; t.s0 = 0.f; t.sb = 0.f; t.x = 0.f; t.diff = 0;
-            if (!dead) {
+            if (!__any_sync(0xffffffffu, dead)) {          // (a lane's own earlier wait may have run out: decide as a warp)
                 bool got = false;
 #pragma unroll 1
-                for (uint32_t i = 0; i < kSpinLimit; ++i) {
+                for (uint32_t i = 0; i < P.poll_limit; ++i) {
+                    // with the first fetch and every 256th: has anybody's wait run out?  (then nothing
+                    // this warp waits for is certain to come, and the group takes no further pair)
+                    const bool look = (i & 255u) == 0;
+                    int gave_up = 0;
+                    if (look && lane == 0) gave_up = *reinterpret_cast<volatile int*>(P.timeout_flag);
                     bool ok = true;
                     if (lane < C) {
                         const uint4 u0 = ld_unit(&xg[par * C + lane].u[0]), u1 = ld_unit(&xg[par * C + lane].u[1]),
@@ -673,8 +680,9 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
                         t.zb = __uint_as_float(u1.x); t.s0 = __uint_as_float(u1.y); t.sb = __uint_as_float(u1.z);
                         t.x = __uint_as_float(u2.x); t.diff = u2.y;
                     }
-                    if (__all_sync(0xffffffffu, ok)) { got = true; break; }
-                    if ((i & 255u) == 255u && *reinterpret_cast<volatile int*>(P.timeout_flag) != 0) break;
+                    const bool all_ok = __all_sync(0xffffffffu, ok);
+                    if (look && __shfl_sync(0xffffffffu, gave_up, 0) != 0) break;
+                    if (all_ok) { got = true; break; }
                 }
                 if (!got) {
                     if (lane == 0) atomicExch(P.timeout_flag, 1);
@@ -683,7 +691,11 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
                 }
             }
             {
-                const uint32_t nxt = __shfl_sync(0xffffffffu, t.diff, 0) >> 1;
+                // after a wait that ran out this group takes no further pair: every member reads the same
+                // "none" and leaves together once the pairs already in its ring are through
+                const uint32_t sent = __shfl_sync(0xffffffffu, t.diff, 0) >> 1;
+                const bool stop = __any_sync(0xffffffffu, dead);
+                const uint32_t nxt = stop ? 0x3fffffffu : sent;
                 t.diff &= 1u;
                 if (lane == 0) sh.items[(li + ahead) & 7] = static_cast<int>(nxt);
             }
