@@ -117,7 +117,11 @@ int fsd_workspace_bytes(int B, int positions, int V, const fsd_opts *opts, size_
  *   row_status    [B] out    FSD_ROW_* flags
  *   workspace     device scratch, 256-byte aligned, at least fsd_workspace_bytes() bytes;
  *                 contents need not be initialised and are not preserved
- * Calls that share a workspace must be ordered on the stream(s) that use it. */
+ * Calls that share a workspace must be ordered on the stream(s) that use it.
+ * The call enqueues a memset and two kernels (the first a cooperative launch of at most one
+ * thread block per SM) and nothing else, so it can be captured in a CUDA graph and replayed --
+ * after one ordinary call with the same options on that device, which sets the kernels'
+ * attributes (that cannot be done under capture). */
 int fsd_verify_chain(const void *target_logits, const void *draft_logits,
                      const int32_t *draft_tokens, const float *u_accept, const float *u_sample,
                      int B, int gamma, int V, const fsd_opts *opts,

@@ -335,3 +335,48 @@ def test_tree_max_depth_and_bad_parent():
         assert g.row_status[1] & 4 and g.accept_len[1] == 0 and g.next_token[1] == -1
         assert g.accept_len.max() <= depth
         parity.compare_divergence(g.divergence, o.divergence, 1e-5)
+
+
+def test_a_verify_call_can_be_captured_in_a_cuda_graph_and_replayed():
+    """A decoding loop captures its steps once and replays them: the call (a memset, the cooperative
+    streaming kernel, the finish kernel) must be capturable after one ordinary call, and a replay on
+    new inputs in the same buffers must give what an ordinary call gives."""
+    import torch
+    from paper_2502_20704_b200 import binding as fsd
+
+    cs = [gi.make_chain(8, 5, 50000, dtype="bf16", recipe="zipf", sigma=(0.3, 1.5), sigma_mode="uniform", workload_id=450 + k)
+          for k in range(2)]
+    want = [parity.check_chain(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, T=0.15)["gpu"] for c in cs]
+    B, g1, V = cs[0].target.shape
+    gamma = g1 - 1
+    opts = fsd.make_opts(dtype="bf16", T=0.15)
+    t = parity.to_device(cs[0].target, "bf16")
+    d = parity.to_device(cs[0].draft, "bf16")
+    us = parity.to_device(cs[0].u_sample, "bf16")
+    acc = torch.zeros(B, dtype=torch.int32, device="cuda")
+    tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+    st = torch.zeros(B, dtype=torch.int32, device="cuda")
+    D = torch.zeros(B, gamma, dtype=torch.float32, device="cuda")
+    wsb = fsd.fsd_workspace_bytes(B, gamma, V, opts)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        assert fsd.fsd_verify_chain(t, d, None, None, us, B, gamma, V, opts, acc, tok, D, st, ws, wsb, side.cuda_stream) == 0
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        rc = fsd.fsd_verify_chain(t, d, None, None, us, B, gamma, V, opts, acc, tok, D, st, ws, wsb, side.cuda_stream)
+    assert rc == 0
+    for k in (1, 0, 1):
+        t.copy_(parity.to_device(cs[k].target, "bf16"))
+        d.copy_(parity.to_device(cs[k].draft, "bf16"))
+        us.copy_(parity.to_device(cs[k].u_sample, "bf16"))
+        acc.fill_(-7); tok.fill_(-7); D.fill_(-7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(acc.cpu().numpy(), want[k].accept_len)
+        assert np.array_equal(tok.cpu().numpy(), want[k].next_token)
+        assert np.array_equal(D.cpu().numpy().view(np.uint32), want[k].divergence.view(np.uint32))
+
