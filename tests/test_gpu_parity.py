@@ -380,3 +380,41 @@ def test_a_verify_call_can_be_captured_in_a_cuda_graph_and_replayed():
         assert np.array_equal(tok.cpu().numpy(), want[k].next_token)
         assert np.array_equal(D.cpu().numpy().view(np.uint32), want[k].divergence.view(np.uint32))
 
+
+def test_calls_of_changing_shapes_queued_on_one_workspace():
+    """Calls of different shapes (so different group sizes, grids and record counts) queued back to
+    back on one stream and one workspace, without a synchronisation in between: nothing one call
+    leaves in the workspace (messages, counters, records) may reach the next.  Each call must give
+    exactly what it gives alone on a fresh workspace."""
+    import torch
+    from paper_2502_20704_b200 import binding as fsd
+
+    shapes = [(3, 4, 32000), (16, 5, 4096), (2, 8, 152064), (40, 3, 8192), (1, 1, 50000), (7, 6, 65544)]
+    cases = [gi.make_chain(B, g, V, dtype="bf16", recipe="zipf", sigma=(0.3, 1.5), sigma_mode="uniform",
+                           disjoint_frac=0.1, workload_id=460 + k) for k, (B, g, V) in enumerate(shapes)]
+    alone = [parity.run_chain_gpu(c.target, c.draft, None, None, c.u_sample, c.dtype, T=0.15) for c in cases]
+    opts = fsd.make_opts(dtype="bf16", T=0.15)
+    wsb = max(fsd.fsd_workspace_bytes(B, g, V, opts) for B, g, V in shapes)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    ws.fill_(0xAB)
+    stream = torch.cuda.current_stream().cuda_stream
+    dev, outs = [], []
+    for c in cases:
+        B, g1, V = c.target.shape
+        dev.append((parity.to_device(c.target, "bf16"), parity.to_device(c.draft, "bf16"), parity.to_device(c.u_sample, "bf16")))
+        outs.append((torch.full((B,), -7, dtype=torch.int32, device="cuda"), torch.full((B,), -7, dtype=torch.int32, device="cuda"),
+                     torch.full((B, g1 - 1), -7.0, dtype=torch.float32, device="cuda"), torch.full((B,), -7, dtype=torch.int32, device="cuda")))
+    torch.cuda.synchronize()
+    order = [0, 1, 2, 3, 4, 5, 5, 2, 0, 4, 3, 1, 2, 2, 4]
+    for k in order:
+        B, g1, V = cases[k].target.shape
+        t, d, us = dev[k]
+        acc, tok, D, st = outs[k]
+        assert fsd.fsd_verify_chain(t, d, None, None, us, B, g1 - 1, V, opts, acc, tok, D, st, ws, wsb, stream) == 0
+    torch.cuda.synchronize()
+    for k, a in enumerate(alone):
+        acc, tok, D, st = outs[k]
+        assert np.array_equal(acc.cpu().numpy(), a.accept_len) and np.array_equal(tok.cpu().numpy(), a.next_token)
+        assert np.array_equal(st.cpu().numpy(), a.row_status)
+        assert np.array_equal(D.cpu().numpy().view(np.uint32), a.divergence.view(np.uint32))
+
