@@ -64,6 +64,7 @@ struct FinishShared {
     int gather_i[2][kMaxClusterSize];
     float kref[kMaxTreeNodes];          // per pair: integer reference at or just above the target row's log2-sum-exp (NaN: none)
     double exp_table[kExpTable];   // 2^(j/256)
+    double exp_consts[8];          // the constants of exp2_table (see exp2_consts)
     double red_d[32 * 2];
     float red_f[32 * 2];
     double warp_tot[32];
@@ -97,6 +98,35 @@ __device__ __forceinline__ double exp2_table(double y, const double* table) {
     const double m = table[k & (kExpTable - 1)] * p;               // in [1, 2.0001)
     const int hi = __double2hiint(m) + ((k >> 8) << 20);           // scale by 2^(k >> 8): stays normal for |y| < 1000
     return __hiloint2double(hi, __double2loint(m));
+}
+
+// The same function, value for value above y = -990 and exactly 0 below about there, for the tight
+// loops of the residual draw: no branch (callers clamp y and say when the result is to be 0; they
+// have excluded NaN), and the constants
+// come as arguments so that a loop keeps them in registers instead of rebuilding each 64-bit
+// immediate at every use.
+struct Exp2Consts { double magic, scale, c4, c3, c2, c1; };
+__device__ __forceinline__ Exp2Consts exp2_consts(const double* opaque) {
+    // read through shared memory: the compiler cannot turn them back into immediates
+    return Exp2Consts{opaque[0], opaque[1], opaque[2], opaque[3], opaque[4], opaque[5]};
+}
+__device__ __forceinline__ double exp2_table_fast(double y, bool below, const double* table, const Exp2Consts& c) {
+    const double t = fma(y, c.scale, c.magic);
+    const int k = __double2loint(t);
+    const double r = fma(y, c.scale, c.magic - t);
+    double p = fma(r, c.c4, c.c3);
+    p = fma(p, r, c.c2);
+    p = fma(p, r, c.c1);
+    p = fma(p, r, 1.0);
+    const double m = table[k & (kExpTable - 1)] * p;
+    const int hi = __double2hiint(m) + ((k >> 8) << 20);
+    return below ? 0.0 : __hiloint2double(hi, __double2loint(m));     // a select, not a branch
+}
+// y = x * log2e - k for the tight loops: x is clamped in single precision at the logit below which
+// y would pass -1000 (`xmin`, with a margin), and `below` tells exp2_table_fast to return exactly 0
+__device__ __forceinline__ double exp2_of_logit(float x, float xmin, double nk, const double* table, const Exp2Consts& c) {
+    const bool below = !(x > xmin);
+    return exp2_table_fast(fma(static_cast<double>(fmaxf(x, xmin)), kLog2eD, nk), below, table, c);
 }
 
 // Every CTA of the cluster publishes a FinishExchange; afterwards sh.all holds everybody's.
@@ -583,6 +613,11 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
 
     // the paths below take their exponentials in double precision from a table
     if (tid < kExpTable) sh.exp_table[tid] = exp2(static_cast<double>(tid) * (1.0 / kExpTable));
+    if (tid == 0) {
+        sh.exp_consts[0] = 6755399441055744.0; sh.exp_consts[1] = 256.0;
+        sh.exp_consts[2] = 2.239395190875157e-12; sh.exp_consts[3] = 3.308302680541371e-09;
+        sh.exp_consts[4] = 3.665565596910106e-06; sh.exp_consts[5] = 2.7076061740622863e-03;
+    }
     __syncthreads();
 
     // ---- references.  A residual draw follows a rejection, so the rejected pair's record has
@@ -657,15 +692,33 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         return;
     }
 
+    // with common references (the usual case): y = x * log2e - k; logits below xmin give 2^y < 2^-990 and count as 0
+    const Exp2Consts ec = exp2_consts(sh.exp_consts);
+    const double nka = -kra, nkb = -krb;
+    const float xmin_a = static_cast<float>((kra - 990.0) * kLn2D), xmin_b = static_cast<float>((krb - 990.0) * kLn2D);
+
     // ---- residual only: global normalisers of both rows (double) ----
     double Ma = Ra, Mb = Rb, iZa = 0.0, iZb = 0.0;
     bool residual = residual0;
     if (residual0) {
         double z[2] = {0.0, 0.0};
+        if (common && vec) {
+            // the usual case (a rejected pair with a record): both rows, two independent exponentials an entry
+            for (int k = k0; k < k1; k += EPV) {
+                float xa[EPV], xb[EPV];
+                unpack_vec<DT>(ldg_vec(a_row, k / EPV), xa);
+                unpack_vec<DT>(ldg_vec(b_row, k / EPV), xb);
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) {
+                    z[0] += exp2_of_logit(xa[e], xmin_a, nka, tab, ec);
+                    z[1] += exp2_of_logit(xb[e], xmin_b, nkb, tab, ec);
+                }
+            }
+        } else
         for_chunk<DT>(a_row, b_row, k0, k1, vec, true, [&](int, float xa, float xb) {
             if (common) {
-                z[0] += exp2_table(fma(static_cast<double>(xa), kLog2eD, -kra), tab);
-                z[1] += exp2_table(fma(static_cast<double>(xb), kLog2eD, -krb), tab);
+                z[0] += exp2_of_logit(xa, xmin_a, nka, tab, ec);
+                z[1] += exp2_of_logit(xb, xmin_b, nkb, tab, ec);
             } else {
                 if (Ra > -INFINITY) z[0] += exp2_table((static_cast<double>(xa) - Ra) * kLog2eD, tab);
                 if (Rb > -INFINITY) z[1] += exp2_table((static_cast<double>(xb) - Rb) * kLog2eD, tab);
@@ -693,10 +746,10 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     for (int attempt = 0; attempt < 2; ++attempt) {
         // weight of one vocabulary entry: P_T relative to this CTA's maximum, or the SD residual
         auto weight = [&](float xa, float xb) -> double {
-            if (common) {
-                const double pa = exp2_table(fma(static_cast<double>(xa), kLog2eD, -kra), tab);
+            if (common) {                                  // the same values as the tight loops
+                const double pa = exp2_of_logit(xa, xmin_a, nka, tab, ec);
                 if (!residual) return pa;
-                const double r = pa * iZa - exp2_table(fma(static_cast<double>(xb), kLog2eD, -krb), tab) * iZb;
+                const double r = pa * iZa - exp2_of_logit(xb, xmin_b, nkb, tab, ec) * iZb;
                 return r > 0.0 ? r : 0.0;
             }
             if (!residual) return Ra > -INFINITY ? exp2_table((static_cast<double>(xa) - Ra) * kLog2eD, tab) : 0.0;
@@ -706,6 +759,20 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         };
         double csum = 0.0, wbest = 0.0;
         int lastp = -1, kbest = 0x7fffffff;
+        if (common && vec && residual && !greedy) {
+            for (int k = k0; k < k1; k += EPV) {
+                float xa[EPV], xb[EPV];
+                unpack_vec<DT>(ldg_vec(a_row, k / EPV), xa);
+                unpack_vec<DT>(ldg_vec(b_row, k / EPV), xb);
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) {
+                    const double pa = exp2_of_logit(xa[e], xmin_a, nka, tab, ec);
+                    const double pb = exp2_of_logit(xb[e], xmin_b, nkb, tab, ec);
+                    const double r = pa * iZa - pb * iZb;
+                    if (r > 0.0) { csum += r; lastp = k + e; }
+                }
+            }
+        } else
         for_chunk<DT>(a_row, b_row, k0, k1, vec, residual, [&](int k, float xa, float xb) {
             const double w = weight(xa, xb);
             csum += w;
