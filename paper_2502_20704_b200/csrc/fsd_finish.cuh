@@ -68,6 +68,7 @@ struct FinishShared {
     double red_d[32 * 2];
     float red_f[32 * 2];
     double warp_tot[32];
+    int amb;                   // residual draw: some entry could not be classed in the first pass
     int cand;                  // lowest thread whose inclusive sum exceeds the target
     int last_pos;              // highest index with a positive weight in this CTA
     int token;
@@ -362,7 +363,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const bool tree = P.parent != nullptr;
 
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");     // "this CTA has started": waited for below
-    if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; sh.token = -1; }
+    if (tid == 0) { sh.cand = 0x7fffffff; sh.last_pos = -1; sh.n_acc = G; sh.bad = 0; sh.row_sel = 0; sh.token = -1; sh.amb = 0; }
     __syncthreads();
     // everything above touched no global memory; what follows reads what the pair kernel wrote
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -625,6 +626,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     //      otherwise one pass for the CTA-local maxima (exact), and for the greedy FSD choice the
     //      argmax of the logits ----
     double kra = 0.0, krb = 0.0;
+    double zea = 0.0, zeb = 0.0;
     bool common = false;
     if (residual0 && P.records != nullptr) {
         const PairRecord* r = P.records + (static_cast<size_t>(b) * G + n);
@@ -636,7 +638,15 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                 nan = nan || a != a || q != q;
                 fa = fmaxf(fa, a); fb = fmaxf(fb, q);
             }
-            if (!nan && isfinite(fa) && isfinite(fb)) { kra = fa; krb = fb; common = true; }
+            if (!nan && isfinite(fa) && isfinite(fb)) {
+                kra = fa; krb = fb; common = true;
+                // the record's (single-precision) normalisers on these references: an estimate of Z_a / Z_b
+                for (uint32_t c = 0; c < r->ncta && c < kMaxGroupSize; ++c) {
+                    const float a = r->part[c].ka, q = r->part[c].kb;
+                    if (a != -INFINITY) zea += static_cast<double>(r->part[c].za) * pow2_int_d(static_cast<double>(a) - fa);
+                    if (q != -INFINITY) zeb += static_cast<double>(r->part[c].zb) * pow2_int_d(static_cast<double>(q) - fb);
+                }
+            }
         }
     }
     float mx[2] = {-INFINITY, -INFINITY};
@@ -700,20 +710,39 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     // ---- residual only: global normalisers of both rows (double) ----
     double Ma = Ra, Mb = Rb, iZa = 0.0, iZb = 0.0;
     bool residual = residual0;
+    // One pass instead of two, where it can be shown to give the same sums.  An entry has residual
+    // weight iff e_a / Z_a > e_b / Z_b, i.e. e_a > rho * e_b with rho = Z_a / Z_b, which is known
+    // only after the pass -- but the record gives rho to about 1e-6.  Entries are classed against
+    // rho_est * (1 +- 1e-4): for those clearly above, e_a and e_b are summed separately, and the
+    // chunk's residual weight is then sum e_a / Z_a - sum e_b / Z_b with the exact normalisers.
+    // An entry between the two bounds (or an estimate that turns out further than 5e-5 off) sends
+    // the whole row through the second pass instead.
+    double sa = 0.0, sb = 0.0;
+    int lastp1 = -1, amb = 0;
+    bool one_pass = false;
     if (residual0) {
         double z[2] = {0.0, 0.0};
         if (common && vec) {
             // the usual case (a rejected pair with a record): both rows, two independent exponentials an entry
+            const bool classify = !greedy && zea > 0.0 && zeb > 0.0 && isfinite(zea) && isfinite(zeb);
+            const double rho_est = classify ? zea / zeb : 0.0;
+            const double rho_hi = rho_est * (1.0 + 1e-4), rho_lo = rho_est * (1.0 - 1e-4);
             for (int k = k0; k < k1; k += EPV) {
                 float xa[EPV], xb[EPV];
                 unpack_vec<DT>(ldg_vec(a_row, k / EPV), xa);
                 unpack_vec<DT>(ldg_vec(b_row, k / EPV), xb);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) {
-                    z[0] += exp2_of_logit(xa[e], xmin_a, nka, tab, ec);
-                    z[1] += exp2_of_logit(xb[e], xmin_b, nkb, tab, ec);
+                    const double pa = exp2_of_logit(xa[e], xmin_a, nka, tab, ec);
+                    const double pb = exp2_of_logit(xb[e], xmin_b, nkb, tab, ec);
+                    z[0] += pa;
+                    z[1] += pb;
+                    if (pa > rho_hi * pb) { sa += pa; sb += pb; lastp1 = k + e; }
+                    else if (!(pa < rho_lo * pb) && pa > 0.0) amb = 1;     // (pa == 0: no weight whatever rho is)
                 }
             }
+            if (!classify) amb = 1;
+            if (amb) atomicOr(&sh.amb, 1);
         } else
         for_chunk<DT>(a_row, b_row, k0, k1, vec, true, [&](int, float xa, float xb) {
             if (common) {
@@ -724,8 +753,8 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                 if (Rb > -INFINITY) z[1] += exp2_table((static_cast<double>(xb) - Rb) * kLog2eD, tab);
             }
         });
-        block_sum<2>(z, sh.red_d);
-        mine.d[0] = Ra; mine.d[1] = Rb; mine.d[2] = z[0]; mine.d[3] = z[1]; mine.i[0] = 0; mine.i[1] = 0;
+        block_sum<2>(z, sh.red_d);                        // (its barriers also order the flag above)
+        mine.d[0] = Ra; mine.d[1] = Rb; mine.d[2] = z[0]; mine.d[3] = z[1]; mine.i[0] = (common && vec) ? sh.amb : 1; mine.i[1] = 0;
         cluster_exchange(cluster, sh, cs, mine);
         Ma = -INFINITY; Mb = -INFINITY;
         for (int r = 0; r < cs; ++r) { Ma = fmax(Ma, all[r].d[0]); Mb = fmax(Mb, all[r].d[1]); }
@@ -741,6 +770,9 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         }
         if (!b_ok) { residual = false; status |= FSD_ROW_NONFINITE; }
         else { iZa = 1.0 / Za; iZb = 1.0 / Zb; }
+        int any_amb = 0;
+        for (int r = 0; r < cs; ++r) any_amb |= all[r].i[0];
+        one_pass = b_ok && any_amb == 0 && fabs(zea * Zb - zeb * Za) <= 5e-5 * zeb * Za;     // |rho_est - rho| <= 5e-5 rho
     }
 
     for (int attempt = 0; attempt < 2; ++attempt) {
@@ -759,7 +791,11 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         };
         double csum = 0.0, wbest = 0.0;
         int lastp = -1, kbest = 0x7fffffff;
-        if (common && vec && residual && !greedy) {
+        if (attempt == 0 && one_pass && residual) {
+            csum = sa * iZa - sb * iZb;
+            if (!(csum > 0.0)) csum = 0.0;
+            lastp = csum > 0.0 ? lastp1 : -1;
+        } else if (common && vec && residual && !greedy) {
             for (int k = k0; k < k1; k += EPV) {
                 float xa[EPV], xb[EPV];
                 unpack_vec<DT>(ldg_vec(a_row, k / EPV), xa);

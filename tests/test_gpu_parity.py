@@ -418,3 +418,29 @@ def test_calls_of_changing_shapes_queued_on_one_workspace():
         assert np.array_equal(st.cpu().numpy(), a.row_status)
         assert np.array_equal(D.cpu().numpy().view(np.uint32), a.divergence.view(np.uint32))
 
+
+def test_residual_draw_when_the_two_rows_agree_almost_everywhere():
+    """SD rule, a rejection between two rows that are identical except for a handful of entries.
+    Every identical entry then has exactly the same weight in both rows and carries residual mass
+    only through the tiny difference of the two normalisers: whether it counts hangs on the exact
+    ratio of the normalisers, which the one-pass form of the residual sums cannot decide from its
+    estimate, so these rows must go through the second pass -- and agree with the oracle there."""
+    rng = np.random.default_rng(471)
+    B, gamma, V = 6, 3, 4096
+    base = (-1.1 * np.log(np.arange(1, V + 1)) + 0.3 * rng.standard_normal((B, gamma + 1, V))).astype(np.float32)
+    target = gi.bf16_bits_to_f32(gi.f32_to_bf16_bits(base))
+    draft = target[:, :gamma, :].copy()
+    tokens = np.zeros((B, gamma), dtype=np.int32)
+    u_acc = np.full((B, gamma), 0.5, dtype=np.float32)
+    for b in range(B):
+        j1, j2 = 1000 + 17 * b, 2000 + 29 * b          # low-probability entries
+        draft[b, 0, j1] += 0.5 * (b + 1)                # q > p there: proposing j1 is rejected for u close to 1
+        draft[b, 0, j2] -= 0.25
+        tokens[b, 0] = j1
+        u_acc[b, 0] = 0.999
+    tbits, dbits = gi.f32_to_bf16_bits(target), gi.f32_to_bf16_bits(draft)
+    u_sample = rng.random(B).astype(np.float32)
+    r = parity.check_chain(tbits, dbits, tokens, u_acc, u_sample, "bf16", mode="sd", T=0.2)
+    assert (r["gpu"].accept_len == 0).all()
+    parity.check_chain(tbits, dbits, tokens, u_acc, u_sample, "bf16", mode="rfsd", T=0.0)
+
