@@ -15,6 +15,11 @@
 // Drawing from the SD residual max(0, P_T - P_D) (Eq. 3) subtracts nearly equal numbers, so
 // there the exponentials are double precision (a 256-entry table times a degree-4 polynomial,
 // about ten fp64 operations) and the sums agree with a sequential double sum to rounding.
+// Usually one pass over the two rows suffices for it: which entries carry residual weight
+// depends on the ratio of the two normalisers only, the rejected pair's record gives that ratio
+// closely enough to class every entry that is not within a margin of the boundary, and the
+// chunk sums follow from the classed sums once the exact normalisers are known; a row with an
+// entry inside the margin takes a second pass.
 #pragma once
 
 #include "fsd_device.cuh"
