@@ -62,8 +62,7 @@ struct FinishExchange {        // what one CTA publishes to its cluster
 constexpr int kExpTable = 256;
 
 struct FinishShared {
-    FinishExchange slot;
-    FinishExchange all[kMaxClusterSize];   // what the cluster's CTAs published (see cluster_exchange)
+    FinishExchange all[2][kMaxClusterSize];   // what the cluster's CTAs published, written by them (see cluster_exchange)
     double sc[kMaxClusterSize];
     double gather_d[2][kMaxClusterSize];   // one value per CTA of the cluster, written by the peers (see cluster_gather)
     int gather_i[2][kMaxClusterSize];
@@ -135,13 +134,13 @@ __device__ __forceinline__ double exp2_of_logit(float x, float xmin, double nk, 
     return exp2_table_fast(fma(static_cast<double>(fmaxf(x, xmin)), kLog2eD, nk), below, table, c);
 }
 
-// Every CTA of the cluster publishes a FinishExchange; afterwards sh.all holds everybody's.
-// Two cluster barriers: after the writes, and after the reads (so the slot can be reused).
-__device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, FinishShared& sh, int cs,
+// Every CTA of the cluster writes a FinishExchange into every CTA's shared memory (its own
+// included); after one cluster barrier sh.all[buf] holds everybody's, in rank order, in every CTA.
+// Like cluster_gather: `buf` alternates from one call to the next, and nobody reads a peer's
+// memory afterwards.  Every thread passes the same `mine`.
+__device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, FinishShared& sh, int cs, int rank, int buf,
                                                  const FinishExchange& mine) {
-    if (threadIdx.x == 0) sh.slot = mine;
-    cluster.sync();
-    if (threadIdx.x < cs) sh.all[threadIdx.x] = cluster.map_shared_rank(&sh, threadIdx.x)->slot;
+    if (threadIdx.x < cs) cluster.map_shared_rank(&sh, threadIdx.x)->all[buf][rank] = mine;
     cluster.sync();
 }
 
@@ -460,7 +459,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     const int k1 = (k0l + L) < V ? static_cast<int>(k0l + L) : V;
     FSD_CHECK(P.debug_word, k0 >= 0 && k0 <= k1 && k1 <= V && (!vec || k0 % EPV == 0), kChkChunk);
     FinishExchange mine;
-    FinishExchange* const all = sh.all;
+    const FinishExchange* all = sh.all[0];
     double* const sc = sh.sc;
 
     // ---- fast path: inverse CDF over P_T (the FSD rule, and every bonus token) ----
@@ -691,7 +690,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         float bv[1] = {bad_v};
         block_max<1>(bv, sh.red_f);
         mine.d[0] = best; mine.d[1] = bv[0]; mine.d[2] = 0; mine.d[3] = 0; mine.i[0] = idx; mine.i[1] = 0;
-        cluster_exchange(cluster, sh, cs, mine);
+        cluster_exchange(cluster, sh, cs, rank, 0, mine);
         double gb = all[0].d[0], gbad = all[0].d[1];
         int gi = all[0].i[0];
         for (int r = 1; r < cs; ++r) {
@@ -760,7 +759,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
         });
         block_sum<2>(z, sh.red_d);                        // (its barriers also order the flag above)
         mine.d[0] = Ra; mine.d[1] = Rb; mine.d[2] = z[0]; mine.d[3] = z[1]; mine.i[0] = (common && vec) ? sh.amb : 1; mine.i[1] = 0;
-        cluster_exchange(cluster, sh, cs, mine);
+        cluster_exchange(cluster, sh, cs, rank, 0, mine);
         Ma = -INFINITY; Mb = -INFINITY;
         for (int r = 0; r < cs; ++r) { Ma = fmax(Ma, all[r].d[0]); Mb = fmax(Mb, all[r].d[1]); }
         double Za = 0.0, Zb = 0.0;
@@ -858,7 +857,8 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             }
         }
         mine.d[0] = cta_tot; mine.d[1] = Ra; mine.d[2] = wbest; mine.d[3] = 0; mine.i[0] = sh.last_pos; mine.i[1] = kbest;
-        cluster_exchange(cluster, sh, cs, mine);
+        cluster_exchange(cluster, sh, cs, rank, 1 - (attempt & 1), mine);
+        all = sh.all[1 - (attempt & 1)];
 
         // cluster totals on a common reference
         double M = -INFINITY;

@@ -3,7 +3,12 @@
 The named workloads fix a handful of shapes; this sweep draws others (vocabulary sizes that are
 and are not multiples of the vector width, group sizes 1 to 16, one to five ring stages per
 pair, masked entries) so that every launch configuration of the pair kernels meets the oracle.
+The number of cases is small by default; FSD_SWEEP_CASES and FSD_SD_SWEEP_CASES in the environment
+extend the two chain sweeps (every case is seeded by its index, so a longer sweep repeats the
+shorter one and goes on).
 """
+
+import os
 
 import numpy as np
 import pytest
@@ -41,7 +46,7 @@ def _case(it: int):
     return c, opts
 
 
-@pytest.mark.parametrize("it", range(24))
+@pytest.mark.parametrize("it", range(int(os.environ.get("FSD_SWEEP_CASES", "24"))))
 def test_random_shape_matches_oracle(it):
     c, opts = _case(it)
     r = parity.check_chain(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, **opts)
@@ -62,3 +67,17 @@ def test_random_tree_matches_oracle(it):
                      max_depth=depth, max_children=children, workload_id=3000 + it)
     parity.check_tree(t, T=float(rng.choice([0.02, 0.1, 0.3, 0.7])), div=str(rng.choice(["js", "kl", "tv"])),
                       cmp=str(rng.choice(["lt", "le"])), sample=str(rng.choice(["invcdf", "greedy"])))
+
+
+@pytest.mark.parametrize("it", range(int(os.environ.get("FSD_SD_SWEEP_CASES", "12"))))
+def test_random_sd_and_rfsd_draws_match_oracle(it):
+    """SD and rFSD only, on larger vocabularies: the residual draw in its one-pass and two-pass forms."""
+    rng = np.random.default_rng(99000 + it)
+    V = int(8 * rng.integers(500, 20000))
+    B, gamma = int(rng.integers(1, 12)), int(rng.integers(1, 8))
+    dtype, recipe = str(rng.choice(["bf16", "f32"])), str(rng.choice(["spike", "zipf"]))
+    c = gi.make_chain(B, gamma, V, dtype=dtype, recipe=recipe, sigma=(0.05, 2.0), sigma_mode="uniform",
+                      disjoint_frac=0.1 if recipe == "zipf" else 0.0, workload_id=7000 + it)
+    parity.check_chain(c.target, c.draft, c.draft_tokens, c.u_accept, c.u_sample, c.dtype, mode=str(rng.choice(["sd", "rfsd"])),
+                       T=float(rng.choice([0.0, 0.05, 0.3])), sample=str(rng.choice(["invcdf", "invcdf", "greedy"])))
+
