@@ -18,8 +18,9 @@
 // Usually one pass over the two rows suffices for it: which entries carry residual weight
 // depends on the ratio of the two normalisers only, the rejected pair's record gives that ratio
 // closely enough to class every entry that is not within a margin of the boundary, and the
-// chunk sums follow from the classed sums once the exact normalisers are known; a row with an
-// entry inside the margin takes a second pass.
+// chunk sums follow from the classed sums once the exact normalisers are known; entries inside
+// the margin are settled one by one afterwards, and a row with too many of them in one thread
+// takes a second pass.
 #pragma once
 
 #include "fsd_device.cuh"
@@ -719,10 +720,11 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
     // only after the pass -- but the record gives rho to about 1e-6.  Entries are classed against
     // rho_est * (1 +- 1e-4): for those clearly above, e_a and e_b are summed separately, and the
     // chunk's residual weight is then sum e_a / Z_a - sum e_b / Z_b with the exact normalisers.
-    // An entry between the two bounds (or an estimate that turns out further than 5e-5 off) sends
-    // the whole row through the second pass instead.
+    // The few entries between the two bounds (about one in 10^4) are remembered, two a thread, and
+    // settled with the exact normalisers afterwards; a thread with more of them, or an estimate
+    // that turns out further than 5e-5 off, sends the whole row through the second pass instead.
     double sa = 0.0, sb = 0.0;
-    int lastp1 = -1, amb = 0;
+    int lastp1 = -1, amb = 0, namb = 0, ak0 = -1, ak1 = -1;
     bool one_pass = false;
     if (residual0) {
         double z[2] = {0.0, 0.0};
@@ -742,10 +744,13 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
                     z[0] += pa;
                     z[1] += pb;
                     if (pa > rho_hi * pb) { sa += pa; sb += pb; lastp1 = k + e; }
-                    else if (!(pa < rho_lo * pb) && pa > 0.0) amb = 1;     // (pa == 0: no weight whatever rho is)
+                    else if (!(pa < rho_lo * pb) && pa > 0.0) {            // (pa == 0: no weight whatever rho is)
+                        if (namb == 0) ak0 = k + e; else ak1 = k + e;
+                        ++namb;
+                    }
                 }
             }
-            if (!classify) amb = 1;
+            if (!classify || namb > 2) amb = 1;
             if (amb) atomicOr(&sh.amb, 1);
         } else
         for_chunk<DT>(a_row, b_row, k0, k1, vec, true, [&](int, float xa, float xb) {
@@ -799,6 +804,12 @@ __global__ void __launch_bounds__(kFinishThreads, 2) fsd_finish_kernel(FinishPar
             csum = sa * iZa - sb * iZb;
             if (!(csum > 0.0)) csum = 0.0;
             lastp = csum > 0.0 ? lastp1 : -1;
+            for (int j = 0; j < namb; ++j) {              // the entries that were too close to call, now with the exact normalisers
+                const int k = j == 0 ? ak0 : ak1;
+                const double r = exp2_of_logit(load_logit<DT>(a_row, k), xmin_a, nka, tab, ec) * iZa -
+                                 exp2_of_logit(load_logit<DT>(b_row, k), xmin_b, nkb, tab, ec) * iZb;
+                if (r > 0.0) { csum += r; lastp = k > lastp ? k : lastp; }
+            }
         } else if (common && vec && residual && !greedy) {
             for (int k = k0; k < k1; k += EPV) {
                 float xa[EPV], xb[EPV];
