@@ -281,14 +281,17 @@ __device__ __forceinline__ void named_sync(int id) {
 }
 constexpr int kBarPosted = 1, kBarTotals = 2;
 
+// One unit is stored and fetched as a single 128-bit access (the .b128 forms: one access, not four
+// that happen to be adjacent), so a reader sees a unit either whole or not at all.
 __device__ __forceinline__ void st_unit(uint4* p, float a, float b, float c, uint32_t tag) {
-    asm volatile("st.relaxed.gpu.global.v4.b32 [%0], {%1, %2, %3, %4};"
-                 ::"l"(p), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)), "r"(tag) : "memory");
+    const uint64_t lo = static_cast<uint64_t>(__float_as_uint(a)) | (static_cast<uint64_t>(__float_as_uint(b)) << 32);
+    const uint64_t hi = static_cast<uint64_t>(__float_as_uint(c)) | (static_cast<uint64_t>(tag) << 32);
+    asm volatile("{ .reg .b128 t; mov.b128 t, {%1, %2}; st.relaxed.gpu.global.b128 [%0], t; }" ::"l"(p), "l"(lo), "l"(hi) : "memory");
 }
 __device__ __forceinline__ uint4 ld_unit(const uint4* p) {
-    uint4 v;
-    asm volatile("ld.relaxed.gpu.global.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
-    return v;
+    uint64_t lo, hi;
+    asm volatile("{ .reg .b128 t; ld.relaxed.gpu.global.b128 t, [%2]; mov.b128 {%0, %1}, t; }" : "=l"(lo), "=l"(hi) : "l"(p) : "memory");
+    return make_uint4(static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi), static_cast<uint32_t>(hi >> 32));
 }
 
 // ---- shared-memory layout ---------------------------------------------------------------
