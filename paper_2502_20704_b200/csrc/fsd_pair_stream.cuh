@@ -423,7 +423,7 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
         if (!live && prev_item < 0) break;
         const int par = static_cast<int>(li & 1);
         const uint32_t tag = li + 1;                 // what this round's messages carry (never 0, the buffer's initial state)
-        if (rank == 0 && lane == 0 && warp == static_cast<int>(li & (kStreamWarps - 1))) {
+        if (kSecondSweep && rank == 0 && lane == 0 && warp == static_cast<int>(li & (kStreamWarps - 1))) {
             // asked now, needed only when the statistics go out
             const long long id = static_cast<long long>(ahead) * n_groups + atomicAdd(P.next_pair, 1);
             claimed = id < 0x3fffffffLL ? static_cast<uint32_t>(id) : 0x3fffffffu;
@@ -651,6 +651,24 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
                 c.x += __shfl_xor_sync(0xffffffffu, c.x, m);
             }
             c.diff = __reduce_or_sync(0xffffffffu, w.diff) != 0 ? 1u : 0u;
+            if constexpr (!kSecondSweep) {
+                // KL has no second sweep, so nobody needs the group's totals: every member leaves its part
+                // straight in the pair's record and goes on.  Without messages there is no channel for
+                // claimed pair ids either: the group's pairs are group_id + round * n_groups throughout.
+                if (live && lane == 0) {
+                    FSD_CHECK(P.timeout_flag + 2, item >= 0 && item < P.n_items && rank < kMaxGroupSize, kChkRecord);
+                    PairRecord* r = P.records + item;
+                    r->part[rank] = c;
+                    if (rank == 0) { r->ncta = static_cast<uint32_t>(C); r->state = bad ? kRecordBadTree : kRecordStats; }
+                }
+                const long long id = static_cast<long long>(group_id) + static_cast<long long>(li + ahead) * n_groups;
+                const bool stop = __any_sync(0xffffffffu, dead);
+                if (lane == 0) {
+                    sh.items[(li + ahead) & 7] = (stop || id >= 0x3fffffffLL) ? 0x3fffffff : static_cast<int>(id);
+                    *reinterpret_cast<float4*>(sh.tot) = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                named_sync(bar_totals);
+            } else {
             {
                 const uint32_t cl = __shfl_sync(0xffffffffu, claimed, 0);   // rank 0's message carries the pair id it took
                 if (rank == 0) c.diff |= cl << 1;
@@ -722,6 +740,7 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
                     if (lane == 0) { r->ncta = static_cast<uint32_t>(C); r->state = bad ? kRecordBadTree : kRecordStats; }
                 }
             }
+            }   // (the exchange that JS and TV need)
         }
         if (warp != static_cast<int>(li & (kStreamWarps - 1))) named_sync(bar_totals);
         const float4 tot = *reinterpret_cast<const float4*>(sh.tot);
@@ -729,7 +748,7 @@ __global__ void __launch_bounds__(kStreamCtaThreads, 1) fsd_pair_stream_kernel(S
         prev_item = -1;
         x_carry = 0.f;
         if (!live) break;
-        prev_item = item;
+        prev_item = kSecondSweep ? item : -1;        // (no second-sweep sum to publish a round later)
 
         // ---- second sweep over the parked e values ----
         if (kSecondSweep) {
